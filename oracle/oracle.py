@@ -1,0 +1,340 @@
+"""ctypes wrapper around the plain-C TapOut oracle (oracle/tapout_oracle.c).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the
+CPU-baseline leg of the benchmark.  It never imports the CUDA package and the
+CUDA package never imports it.  Arrays are numpy; logits are float32 arrays or
+uint16 arrays holding bf16 bit patterns.
+"""
+import ctypes as C
+
+import numpy as np
+
+from . import build as _build
+
+FP32, BF16 = 0, 1
+UCB1, TS, UCB_TUNED = 0, 1, 2
+SEQ, TOKEN = 0, 1
+RULE_MAXCONF, RULE_SVIP, RULE_ADAEDL, RULE_SVIPDIFF, RULE_MARGIN, RULE_STATIC = range(6)
+RNG_DRAFT, RNG_ACCEPT, RNG_RESAMPLE, RNG_BANDIT = range(4)
+ST_BAD_DRAFT_ROW, ST_BAD_TARGET_ROW, ST_ZERO_RESIDUAL = 1, 2, 4
+
+_lib = None
+
+
+class RowStats(C.Structure):
+    _fields_ = [("m", C.c_double), ("W", C.c_double), ("lse", C.c_double), ("p1", C.c_double),
+                ("p2", C.c_double), ("H", C.c_double), ("argmax", C.c_int), ("valid", C.c_int)]
+
+
+class RuleParams(C.Structure):
+    _fields_ = [("h_maxconf", C.c_double), ("h_svip", C.c_double), ("h_diff", C.c_double),
+                ("h_margin", C.c_double), ("ada_gamma", C.c_double), ("ada_alpha", C.c_double),
+                ("ada_beta1", C.c_double), ("ada_beta2", C.c_double), ("ada_eps", C.c_double)]
+
+    @classmethod
+    def default(cls):
+        return cls(0.8, 0.6, 0.2, 0.2, 0.2, 0.9, 0.5, 0.9, 0.01)
+
+
+class VerifyOut(C.Structure):
+    _fields_ = [("accept_len", C.c_int), ("next_token", C.c_int), ("next_lo", C.c_int),
+                ("next_hi", C.c_int), ("near_accept", C.c_int), ("zero_residual", C.c_int),
+                ("bad_target", C.c_int), ("ratio_at_stop", C.c_double)]
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(_build.build())
+        vp, u32, u64, i32, dbl = C.c_void_p, C.c_uint32, C.c_uint64, C.c_int, C.c_double
+        L.orc_philox4x32_10.argtypes = [vp, vp, vp]
+        L.orc_rng_u24.restype = u32
+        L.orc_rng_u24.argtypes = [u64, u32, u32, u32, u32, u32, u32, i32]
+        L.orc_rng_uniform.restype = dbl
+        L.orc_rng_uniform.argtypes = [u64, u32, u32, u32, u32, u32, u32, i32]
+        L.orc_row_stats.argtypes = [vp, i32, i32, C.c_float, vp, C.POINTER(RowStats)]
+        L.orc_sample_cdf.argtypes = [vp, i32, dbl, dbl, dbl, C.POINTER(i32), C.POINTER(i32)]
+        L.orc_rule_stop.argtypes = [i32, dbl, dbl, dbl, dbl, i32, dbl, C.POINTER(RuleParams), dbl, C.POINTER(i32)]
+        L.orc_adaedl_update.argtypes = [C.POINTER(dbl), C.POINTER(dbl), i32, i32, C.POINTER(RuleParams)]
+        L.orc_reward_simple.restype = dbl
+        L.orc_reward_simple.argtypes = [i32, i32]
+        L.orc_reward_blend.restype = dbl
+        L.orc_reward_blend.argtypes = [i32, i32, i32, dbl]
+        L.orc_ucb1_select.argtypes = [vp, vp, i32, dbl, dbl, vp, C.POINTER(u32)]
+        L.orc_ucb_tuned_select.argtypes = [vp, vp, vp, i32, dbl, vp, C.POINTER(u32)]
+        L.orc_ts_gauss_select.argtypes = [vp, vp, i32, dbl, dbl, dbl, u64, u32, u32, u32, dbl, vp, C.POINTER(u32)]
+        L.orc_beta_order_stat.restype = u32
+        L.orc_beta_order_stat.argtypes = [u32, u32, u64, u32, u32, u32, u32]
+        L.orc_ts_beta_select.argtypes = [vp, vp, i32, u32, u32, u64, u32, u32, u32, vp]
+        L.orc_verify_sequence.argtypes = [vp, C.c_long, vp, C.c_long, i32, i32, C.c_float, C.c_float,
+                                          vp, i32, vp, u64, u32, u32, dbl, vp, C.POINTER(VerifyOut)]
+        L.orc_create.restype = vp
+        L.orc_create.argtypes = [i32] * 6
+        L.orc_destroy.argtypes = [vp]
+        L.orc_draft_step.argtypes = [vp, vp, C.c_long, vp, vp, vp, vp, vp, vp]
+        L.orc_verify.argtypes = [vp, vp, C.c_long, C.c_long, vp, C.c_long, C.c_long, vp, vp, vp, vp, vp, vp]
+        L.orc_update.argtypes = [vp]
+        L.orc_set_param.argtypes = [vp, C.c_char_p, dbl]
+        L.orc_set_seed.argtypes = [vp, u64]
+        L.orc_get_P.argtypes = [vp]
+        L.orc_get_round.restype = u32
+        L.orc_get_round.argtypes = [vp]
+        L.orc_get_pos.argtypes = [vp]
+        L.orc_get_status.restype = u64
+        L.orc_get_status.argtypes = [vp]
+        L.orc_get_rows.restype = u64
+        L.orc_get_rows.argtypes = [vp]
+        for f in ("seq_id", "cnt", "rsum", "rsum2", "lambda", "acc_rate", "arm", "n_drafted", "active",
+                  "void_round", "sqrtH_prev", "lse_q", "feat", "accept_len", "reward", "rule_of_arm"):
+            fn = getattr(L, "orc_ptr_" + f)
+            fn.restype = vp
+            fn.argtypes = [vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _dtype_code(row):
+    if row.dtype == np.float32:
+        return FP32
+    if row.dtype == np.uint16:
+        return BF16
+    raise TypeError("logits must be float32 or uint16 (bf16 bits), got %s" % row.dtype)
+
+
+# ---------------------------------------------------------------- primitives
+def philox4x32_10(ctr, key):
+    c = np.asarray(ctr, dtype=np.uint32)
+    k = np.asarray(key, dtype=np.uint32)
+    out = np.zeros(4, dtype=np.uint32)
+    lib().orc_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def rng_u24(seed, seq, rnd, pos, purpose, arm=0, draw=0, word=0):
+    return int(lib().orc_rng_u24(seed, seq, rnd, pos, purpose, arm, draw, word))
+
+
+def rng_uniform(seed, seq, rnd, pos, purpose, arm=0, draw=0, word=0):
+    return float(lib().orc_rng_uniform(seed, seq, rnd, pos, purpose, arm, draw, word))
+
+
+def row_stats(row, inv_T=1.0, want_w=False):
+    row = np.ascontiguousarray(row)
+    st = RowStats()
+    w = np.zeros(row.shape[0], dtype=np.float64) if want_w else None
+    lib().orc_row_stats(_ptr(row), _dtype_code(row), row.shape[0], np.float32(inv_T), _ptr(w), C.byref(st))
+    return (st, w) if want_w else st
+
+
+def sample_cdf(w, total, u, tol=1e-6):
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    lo, hi = C.c_int(), C.c_int()
+    x = lib().orc_sample_cdf(_ptr(w), w.shape[0], total, u, tol, C.byref(lo), C.byref(hi))
+    return x, lo.value, hi.value
+
+
+def rule_stop(rule, p1, p2, H, sqrtH_prev=0.0, has_prev=0, lam=0.4, rp=None, tol=1e-6):
+    rp = rp or RuleParams.default()
+    near = C.c_int()
+    stop = lib().orc_rule_stop(rule, p1, p2, H, sqrtH_prev, has_prev, lam, C.byref(rp), tol, C.byref(near))
+    return bool(stop), bool(near.value)
+
+
+def adaedl_update(lam, acc, n_acc, n_drafted, rp=None):
+    rp = rp or RuleParams.default()
+    l, a = C.c_double(lam), C.c_double(acc)
+    lib().orc_adaedl_update(C.byref(l), C.byref(a), n_acc, n_drafted, C.byref(rp))
+    return l.value, a.value
+
+
+def reward_simple(n_acc, gamma):
+    return lib().orc_reward_simple(n_acc, gamma)
+
+
+def reward_blend(n_acc, n_drafted, gamma, alpha=0.5):
+    return lib().orc_reward_blend(n_acc, n_drafted, gamma, alpha)
+
+
+def ucb1_select(N, R, c2=2.0, tol=1e-6):
+    N = np.ascontiguousarray(N, dtype=np.uint32)
+    R = np.ascontiguousarray(R, dtype=np.float64)
+    idx = np.zeros(N.shape[0])
+    mk = C.c_uint32()
+    a = lib().orc_ucb1_select(_ptr(N), _ptr(R), N.shape[0], c2, tol, _ptr(idx), C.byref(mk))
+    return a, idx, mk.value
+
+
+def ucb_tuned_select(N, R, R2, tol=1e-6):
+    N = np.ascontiguousarray(N, dtype=np.uint32)
+    R = np.ascontiguousarray(R, dtype=np.float64)
+    R2 = np.ascontiguousarray(R2, dtype=np.float64)
+    idx = np.zeros(N.shape[0])
+    mk = C.c_uint32()
+    a = lib().orc_ucb_tuned_select(_ptr(N), _ptr(R), _ptr(R2), N.shape[0], tol, _ptr(idx), C.byref(mk))
+    return a, idx, mk.value
+
+
+def ts_gauss_select(N, R, seed, seq, rnd, pos=0, mu0=0.0, var0=1.0, noise_var=1.0, tol=1e-6):
+    N = np.ascontiguousarray(N, dtype=np.uint32)
+    R = np.ascontiguousarray(R, dtype=np.float64)
+    smp = np.zeros(N.shape[0])
+    mk = C.c_uint32()
+    a = lib().orc_ts_gauss_select(_ptr(N), _ptr(R), N.shape[0], mu0, var0, noise_var, seed, seq, rnd, pos,
+                                  tol, _ptr(smp), C.byref(mk))
+    return a, smp, mk.value
+
+
+def beta_order_stat(alpha, beta, seed, seq, rnd, pos, arm):
+    return int(lib().orc_beta_order_stat(alpha, beta, seed, seq, rnd, pos, arm))
+
+
+def ts_beta_select(N, R, seed, seq, rnd, pos, a0=1, b0=1):
+    N = np.ascontiguousarray(N, dtype=np.uint32)
+    R = np.ascontiguousarray(R, dtype=np.float64)
+    smp = np.zeros(N.shape[0], dtype=np.uint32)
+    a = lib().orc_ts_beta_select(_ptr(N), _ptr(R), N.shape[0], a0, b0, seed, seq, rnd, pos, _ptr(smp))
+    return a, smp
+
+
+def verify_sequence(q_rows, p_rows, x, lse_q, seed, seq, rnd, inv_Tq=1.0, inv_Tp=1.0, tol=1e-6):
+    """q_rows [n][V] (or more rows), p_rows [>= n+1][V], x [n] tokens, lse_q [n]."""
+    q_rows = np.ascontiguousarray(q_rows)
+    p_rows = np.ascontiguousarray(p_rows)
+    x = np.ascontiguousarray(x, dtype=np.int32)
+    lse_q = np.ascontiguousarray(lse_q, dtype=np.float64)
+    V = p_rows.shape[1]
+    scratch = np.zeros(3 * V)
+    out = VerifyOut()
+    lib().orc_verify_sequence(_ptr(q_rows), V, _ptr(p_rows), V, _dtype_code(p_rows), V,
+                              np.float32(inv_Tq), np.float32(inv_Tp), _ptr(x), x.shape[0], _ptr(lse_q),
+                              seed, seq, rnd, tol, _ptr(scratch), C.byref(out))
+    return out
+
+
+# -------------------------------------------------------------------- engine
+class Oracle:
+    """Algorithm 1 over a batch of independent sequences, on host arrays."""
+
+    def __init__(self, n_seq, vocab, k_max, n_arms, policy, level, **params):
+        self.L = lib()
+        self.S, self.V, self.K, self.A = n_seq, vocab, k_max, n_arms
+        self.policy, self.level = policy, level
+        self.h = self.L.orc_create(n_seq, vocab, k_max, n_arms, policy, level)
+        if not self.h:
+            raise ValueError("orc_create rejected the arguments")
+        self.P = self.L.orc_get_P(self.h)
+        for k, v in params.items():
+            self.set_param(k, v)
+
+    def close(self):
+        if self.h:
+            self.L.orc_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_param(self, key, value):
+        if key == "seed":
+            self.L.orc_set_seed(self.h, int(value))
+            return
+        if key == "seq_ids":
+            self.view("seq_id")[:] = np.asarray(value, dtype=np.uint32)
+            return
+        if key == "arms":
+            r = self.view("rule_of_arm")
+            r[: len(value)] = np.asarray(value, dtype=np.int32)
+            return
+        if self.L.orc_set_param(self.h, key.encode(), float(value)) != 0:
+            raise KeyError(key)
+
+    _FIELDS = {
+        "seq_id": (np.uint32, lambda o: (o.S,)),
+        "cnt": (np.uint32, lambda o: (o.S, o.P, o.A)),
+        "rsum": (np.float64, lambda o: (o.S, o.P, o.A)),
+        "rsum2": (np.float64, lambda o: (o.S, o.P, o.A)),
+        "lambda": (np.float64, lambda o: (o.S,)),
+        "acc_rate": (np.float64, lambda o: (o.S,)),
+        "arm": (np.int32, lambda o: (o.S, o.K)),
+        "n_drafted": (np.int32, lambda o: (o.S,)),
+        "active": (np.uint8, lambda o: (o.S,)),
+        "void_round": (np.uint8, lambda o: (o.S,)),
+        "sqrtH_prev": (np.float64, lambda o: (o.S,)),
+        "lse_q": (np.float64, lambda o: (o.S, o.K)),
+        "feat": (np.float64, lambda o: (o.S, o.K, 6)),
+        "accept_len": (np.int32, lambda o: (o.S,)),
+        "reward": (np.float64, lambda o: (o.S,)),
+        "rule_of_arm": (np.int32, lambda o: (16,)),
+    }
+
+    def view(self, name):
+        """Live numpy view of one of the engine's arrays."""
+        dt, shp = self._FIELDS[name]
+        shape = shp(self)
+        addr = getattr(self.L, "orc_ptr_" + name)(self.h)
+        n = int(np.prod(shape))
+        buf = (C.c_char * (n * np.dtype(dt).itemsize)).from_address(addr)
+        return np.frombuffer(buf, dtype=dt).reshape(shape)
+
+    @property
+    def round(self):
+        return int(self.L.orc_get_round(self.h))
+
+    @property
+    def pos(self):
+        return int(self.L.orc_get_pos(self.h))
+
+    @property
+    def status(self):
+        return int(self.L.orc_get_status(self.h))
+
+    @property
+    def rows_read(self):
+        return int(self.L.orc_get_rows(self.h))
+
+    def draft_step(self, logits, row_stride=None):
+        """logits: array whose row s starts row_stride elements after row s-1."""
+        S = self.S
+        tok = np.empty(S, np.int32)
+        cont = np.empty(S, np.uint8)
+        lo = np.empty(S, np.int32)
+        hi = np.empty(S, np.int32)
+        near = np.empty(S, np.uint8)
+        mask = np.empty(S, np.uint32)
+        if row_stride is None:
+            assert logits.ndim == 2 and logits.shape == (S, self.V)
+            row_stride = logits.strides[0] // logits.itemsize
+        rc = self.L.orc_draft_step(self.h, logits.ctypes.data, row_stride, _ptr(tok), _ptr(cont),
+                                   _ptr(lo), _ptr(hi), _ptr(near), _ptr(mask))
+        if rc != 0:
+            raise RuntimeError("orc_draft_step: bad call order (%d)" % rc)
+        return dict(token=tok, cont=cont, tok_lo=lo, tok_hi=hi, near_rule=near, arm_mask=mask)
+
+    def verify(self, draft_logits, target_logits, draft_tokens):
+        """draft_logits [S][K][V], target_logits [S][K+1][V] (C-contiguous), draft_tokens [S][K]."""
+        S, K, V = self.S, self.K, self.V
+        assert draft_logits.shape == (S, K, V) and target_logits.shape == (S, K + 1, V)
+        assert draft_logits.flags.c_contiguous and target_logits.flags.c_contiguous
+        dt = np.ascontiguousarray(draft_tokens, dtype=np.int32)
+        acc = np.empty(S, np.int32)
+        nxt = np.empty(S, np.int32)
+        lo = np.empty(S, np.int32)
+        hi = np.empty(S, np.int32)
+        near = np.empty(S, np.uint8)
+        rc = self.L.orc_verify(self.h, draft_logits.ctypes.data, K * V, V, target_logits.ctypes.data,
+                               (K + 1) * V, V, _ptr(dt), _ptr(acc), _ptr(nxt), _ptr(lo), _ptr(hi), _ptr(near))
+        if rc != 0:
+            raise RuntimeError("orc_verify: bad call order (%d)" % rc)
+        return dict(accept_len=acc, next_token=nxt, next_lo=lo, next_hi=hi, near_accept=near)
+
+    def update(self):
+        rc = self.L.orc_update(self.h)
+        if rc != 0:
+            raise RuntimeError("orc_update: bad call order (%d)" % rc)

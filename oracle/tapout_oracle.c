@@ -1,0 +1,765 @@
+/*
+ * TapOut oracle: plain, slow, double-precision CPU implementation.
+ *
+ * TEST INFRASTRUCTURE ONLY. This file is the parity reference for the CUDA
+ * library; it shares no code with it and the product never calls it.  Every
+ * function restates one passage of the TapOut paper (arXiv 2511.02017) in the
+ * paper's order and notation, one loop per formula, no blocking or fusion.
+ *
+ * Passages followed
+ *   Algorithm 1          : draft loop / stop query / verify / final token / update
+ *   Section 3.2          : rewards r_simple, r_blend (alpha = 0.5), token-level 0/1
+ *   Section 3.3          : UCB1 index, UCB-Tuned index, Thompson Sampling
+ *                          (Beta-Bernoulli at token level, Gaussian at sequence level)
+ *   Table 1, Appendix A.1: the five stop rules and the AdaEDL lambda update
+ *   Section 1 (refs)     : speculative sampling, accept with prob min(1, p/q),
+ *                          resample from norm(max(0, p - q)), bonus token from p
+ *
+ * Where the paper is silent the reading taken is written next to the code.
+ * Randomness is Philox4x32-10 (Salmon et al. 2011) keyed by
+ * (seed, sequence, round, position, purpose); uniforms carry 24 bits so they
+ * are exact in float and double.
+ *
+ * All pins live in tests/ (closed forms, brute force, library routines,
+ * published Philox vectors, chi-square on tiny vocabularies).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_FP32 0
+#define ORC_BF16 1
+
+#define ORC_UCB1 0
+#define ORC_TS 1
+#define ORC_UCB_TUNED 2
+
+#define ORC_SEQ 0
+#define ORC_TOKEN 1
+
+/* rule ids, Table 1 in table order */
+#define ORC_RULE_MAXCONF 0
+#define ORC_RULE_SVIP 1
+#define ORC_RULE_ADAEDL 2
+#define ORC_RULE_SVIPDIFF 3
+#define ORC_RULE_MARGIN 4
+#define ORC_RULE_STATIC 5 /* never stops early (fixed-length drafting, the Static-k baseline) */
+
+/* Philox purposes */
+#define ORC_RNG_DRAFT 0
+#define ORC_RNG_ACCEPT 1
+#define ORC_RNG_RESAMPLE 2
+#define ORC_RNG_BANDIT 3
+
+/* status bits */
+#define ORC_ST_BAD_DRAFT_ROW 1ull
+#define ORC_ST_BAD_TARGET_ROW 2ull
+#define ORC_ST_ZERO_RESIDUAL 4ull
+
+#define ORC_MAX_ARMS 16
+
+/* ------------------------------------------------------------------------- */
+/* Philox4x32-10, as published (Salmon, Moraes, Dror, Shaw, SC'11).          */
+/* ------------------------------------------------------------------------- */
+void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u; /* multipliers */
+    const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u; /* Weyl key increments */
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int r = 0; r < 10; ++r) {
+        uint64_t p0 = (uint64_t)M0 * c0;
+        uint64_t p1 = (uint64_t)M1 * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += W0; k1 += W1;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* counter = (sequence id, round, position, purpose | arm << 4 | draw << 8),
+ * key = the 64-bit seed.  Returns the four raw words. */
+void orc_rng_words(uint64_t seed, uint32_t seq, uint32_t round, uint32_t pos,
+                   uint32_t purpose, uint32_t arm, uint32_t draw, uint32_t out[4])
+{
+    uint32_t ctr[4] = { seq, round, pos, (purpose & 15u) | ((arm & 15u) << 4) | (draw << 8) };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    orc_philox4x32_10(ctr, key, out);
+}
+
+/* 24-bit integer uniform and its value in [0,1). */
+uint32_t orc_rng_u24(uint64_t seed, uint32_t seq, uint32_t round, uint32_t pos,
+                     uint32_t purpose, uint32_t arm, uint32_t draw, int word)
+{
+    uint32_t w[4];
+    orc_rng_words(seed, seq, round, pos, purpose, arm, draw, w);
+    return w[word & 3] >> 8;
+}
+
+double orc_rng_uniform(uint64_t seed, uint32_t seq, uint32_t round, uint32_t pos,
+                       uint32_t purpose, uint32_t arm, uint32_t draw, int word)
+{
+    return (double)orc_rng_u24(seed, seq, round, pos, purpose, arm, draw, word) * (1.0 / 16777216.0);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Logit rows.                                                               */
+/* ------------------------------------------------------------------------- */
+static double load_logit(const void* row, int dtype, long v)
+{
+    if (dtype == ORC_FP32) return (double)((const float*)row)[v];
+    uint32_t bits = ((uint32_t)((const uint16_t*)row)[v]) << 16; /* bf16 = top half of a float */
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return (double)f;
+}
+
+typedef struct {
+    double m;     /* max_v s_v, s_v = z_v * inv_T                       */
+    double W;     /* sum_v exp(s_v - m)                                 */
+    double lse;   /* m + ln W                                           */
+    double p1;    /* largest softmax probability                        */
+    double p2;    /* second largest, by element (a tie gives p2 == p1)  */
+    double H;     /* entropy in nats                                    */
+    int argmax;   /* lowest index attaining the maximum                 */
+    int valid;    /* 0: NaN present, or no finite maximum               */
+} orc_rowstats;
+
+/* Softmax statistics of one row (features of Table 1).  w_out, if not NULL,
+ * receives w_v = exp(s_v - m) for all v.  Returns st->valid. */
+int orc_row_stats(const void* row, int dtype, int V, float inv_T, double* w_out, orc_rowstats* st)
+{
+    double t = (double)inv_T;
+    memset(st, 0, sizeof *st);
+    st->argmax = -1;
+    if (V <= 0) return 0;
+
+    double m = -INFINITY;
+    int arg = -1, has_nan = 0;
+    for (int v = 0; v < V; ++v) {
+        double s = load_logit(row, dtype, v) * t;
+        if (isnan(s)) has_nan = 1;
+        if (s > m) { m = s; arg = v; }
+    }
+    if (has_nan || !isfinite(m)) { st->m = m; return 0; }
+
+    double W = 0.0;
+    for (int v = 0; v < V; ++v) {
+        double w = exp(load_logit(row, dtype, v) * t - m);
+        if (w_out) w_out[v] = w;
+        W += w;
+    }
+    double lse = m + log(W);
+
+    double p1 = -1.0, p2 = -1.0, H = 0.0;
+    for (int v = 0; v < V; ++v) {
+        double s = load_logit(row, dtype, v) * t;
+        double q = (w_out ? w_out[v] : exp(s - m)) / W;   /* softmax probability */
+        if (q > p1) { p2 = p1; p1 = q; }
+        else if (q > p2) { p2 = q; }
+        if (q > 0.0) H -= q * (s - lse);    /* ln q_v = s_v - lse, so -q ln q     */
+    }
+    if (p2 < 0.0) p2 = 0.0;                 /* V == 1 */
+    if (H < 0.0) H = 0.0;
+
+    st->m = m; st->W = W; st->lse = lse; st->p1 = p1; st->p2 = p2; st->H = H;
+    st->argmax = arg; st->valid = 1;
+    return 1;
+}
+
+/* Inverse-CDF draw in token-index order: the first j whose running sum
+ * c_j = sum_{v<=j} w_v exceeds u * total; if rounding leaves none, the last j
+ * with w_j > 0.  lo/hi (optional) are the draws for (u - tol) and (u + tol):
+ * every token between them with positive weight is an answer a computation
+ * with relative error tol in the sums could legitimately give. */
+static int first_exceeding(const double* w, int V, double target)
+{
+    double c = 0.0;
+    int last_pos = -1;
+    for (int j = 0; j < V; ++j) {
+        if (w[j] > 0.0) last_pos = j;
+        c += w[j];
+        if (c > target) return j;
+    }
+    return last_pos;
+}
+
+int orc_sample_cdf(const double* w, int V, double total, double u, double tol, int* lo, int* hi)
+{
+    int x = first_exceeding(w, V, u * total);
+    if (lo) { double ul = u - tol; if (ul < 0.0) ul = 0.0; *lo = first_exceeding(w, V, ul * total); }
+    if (hi) *hi = first_exceeding(w, V, (u + tol) * total);
+    return x;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Stop rules, Table 1 / Appendix A.1.  Strict inequalities as printed.      */
+/* ------------------------------------------------------------------------- */
+typedef struct {
+    double h_maxconf;   /* 0.8 */
+    double h_svip;      /* 0.6 */
+    double h_diff;      /* 0.2 */
+    double h_margin;    /* 0.2 */
+    double ada_gamma, ada_alpha, ada_beta1, ada_beta2, ada_eps; /* AdaEDL's own symbols */
+} orc_ruleparams;
+
+/* Returns 1 = stop.  sqrtH_prev is sqrt(H) of the previous draft position of
+ * this round; has_prev = 0 at the first position (no previous draft
+ * distribution exists, so SVIPDifference continues).  *near (optional) is set
+ * when the compared quantity lies within tol of its threshold. */
+int orc_rule_stop(int rule, double p1, double p2, double H, double sqrtH_prev, int has_prev,
+                  double lambda, const orc_ruleparams* rp, double tol, int* near)
+{
+    double lhs = 0.0, rhs = 0.0;
+    int stop = 0, applicable = 1;
+    switch (rule) {
+    case ORC_RULE_MAXCONF:  lhs = p1;                              rhs = rp->h_maxconf; stop = lhs < rhs; break;
+    case ORC_RULE_SVIP:     lhs = sqrt(H);                         rhs = rp->h_svip;    stop = lhs > rhs; break;
+    case ORC_RULE_ADAEDL:   lhs = 1.0 - sqrt(rp->ada_gamma * H);   rhs = lambda;        stop = lhs < rhs; break;
+    case ORC_RULE_SVIPDIFF:
+        if (!has_prev) { applicable = 0; stop = 0; break; }
+        lhs = sqrt(H) - sqrtH_prev;                                rhs = rp->h_diff;    stop = lhs > rhs; break;
+    case ORC_RULE_MARGIN:   lhs = p1 - p2;                         rhs = rp->h_margin;  stop = lhs < rhs; break;
+    default:                applicable = 0; stop = 0; break;       /* ORC_RULE_STATIC */
+    }
+    if (near) *near = applicable && fabs(lhs - rhs) <= tol;
+    return stop;
+}
+
+/* AdaEDL update after each full draft (Appendix A.1), as printed:
+ *   r = n_acc / n_drafted
+ *   accept_rate <- beta1 * accept_rate + (1 - beta1) * r
+ *   lambda      <- beta2 * lambda + (1 - beta2) * (lambda + eps * sign(alpha - r)) */
+void orc_adaedl_update(double* lambda, double* accept_rate, int n_acc, int n_drafted, const orc_ruleparams* rp)
+{
+    double r = (double)n_acc / (double)n_drafted;
+    double d = rp->ada_alpha - r;
+    double sgn = (d > 0.0) - (d < 0.0);
+    *accept_rate = rp->ada_beta1 * (*accept_rate) + (1.0 - rp->ada_beta1) * r;
+    *lambda = rp->ada_beta2 * (*lambda) + (1.0 - rp->ada_beta2) * ((*lambda) + rp->ada_eps * sgn);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Rewards, Section 3.2.                                                     */
+/* ------------------------------------------------------------------------- */
+double orc_reward_simple(int n_acc, int gamma) { return (double)n_acc / (double)gamma; }
+
+double orc_reward_blend(int n_acc, int n_drafted, int gamma, double alpha)
+{
+    return alpha * ((double)n_acc / (double)gamma) + (1.0 - alpha) * ((double)n_acc / (double)n_drafted);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Bandits, Section 3.3.                                                     */
+/* ------------------------------------------------------------------------- */
+/* Picks the arm with the largest value, ties to the lowest index; *near_mask
+ * (optional) gets a bit for every arm whose value is within tol of the best. */
+static int argmax_first(const double* val, int A, double tol, uint32_t* near_mask)
+{
+    int best = 0;
+    for (int a = 1; a < A; ++a) if (val[a] > val[best]) best = a;
+    if (near_mask) {
+        uint32_t mk = 0;
+        for (int a = 0; a < A; ++a) if (val[best] - val[a] <= tol) mk |= 1u << a;
+        *near_mask = mk;
+    }
+    return best;
+}
+
+/* UCB1: argmax_a mu_a + sqrt(c2 * ln t / N_a), c2 = 2 as printed.  N_a counts
+ * plays before time t, so t = 1 + sum_a N_a.  An arm never played has an
+ * unbounded bonus: unplayed arms are tried first, in index order. */
+int orc_ucb1_select(const uint32_t* N, const double* R, int A, double c2, double tol,
+                    double* index_out, uint32_t* near_mask)
+{
+    for (int a = 0; a < A; ++a)
+        if (N[a] == 0) { if (near_mask) *near_mask = 1u << a; if (index_out) for (int b = 0; b < A; ++b) index_out[b] = (N[b] == 0) ? INFINITY : 0.0; return a; }
+    uint64_t t = 1;
+    for (int a = 0; a < A; ++a) t += N[a];
+    double lt = log((double)t);
+    double val[ORC_MAX_ARMS];
+    for (int a = 0; a < A; ++a) {
+        double mu = R[a] / (double)N[a];
+        val[a] = mu + sqrt(c2 * lt / (double)N[a]);
+        if (index_out) index_out[a] = val[a];
+    }
+    return argmax_first(val, A, tol, near_mask);
+}
+
+/* UCB-Tuned: mu_a + sqrt( (ln t / N_a) * min(1/4, V_a) ),
+ * V_a = sigma2_a + sqrt(2 ln t / N_a), sigma2_a = empirical variance
+ * (mean of squares minus square of mean). */
+int orc_ucb_tuned_select(const uint32_t* N, const double* R, const double* R2, int A, double tol,
+                         double* index_out, uint32_t* near_mask)
+{
+    for (int a = 0; a < A; ++a)
+        if (N[a] == 0) { if (near_mask) *near_mask = 1u << a; if (index_out) for (int b = 0; b < A; ++b) index_out[b] = (N[b] == 0) ? INFINITY : 0.0; return a; }
+    uint64_t t = 1;
+    for (int a = 0; a < A; ++a) t += N[a];
+    double lt = log((double)t);
+    double val[ORC_MAX_ARMS];
+    for (int a = 0; a < A; ++a) {
+        double n = (double)N[a];
+        double mu = R[a] / n;
+        double var = R2[a] / n - mu * mu;
+        double Va = var + sqrt(2.0 * lt / n);
+        double cap = Va < 0.25 ? Va : 0.25;
+        val[a] = mu + sqrt((lt / n) * cap);
+        if (index_out) index_out[a] = val[a];
+    }
+    return argmax_first(val, A, tol, near_mask);
+}
+
+/* Thompson Sampling, Gaussian prior N(mu0, var0) with known noise variance
+ * (sequence level).  Conjugate posterior after N plays with reward sum R:
+ *   var_n = 1 / (1/var0 + N/noise),  mu_n = var_n * (mu0/var0 + R/noise).
+ * One Box-Muller normal per arm from two 24-bit uniforms of one Philox call. */
+int orc_ts_gauss_select(const uint32_t* N, const double* R, int A,
+                        double mu0, double var0, double noise_var,
+                        uint64_t seed, uint32_t seq, uint32_t round, uint32_t pos,
+                        double tol, double* sample_out, uint32_t* near_mask)
+{
+    double val[ORC_MAX_ARMS];
+    for (int a = 0; a < A; ++a) {
+        double var_n = 1.0 / (1.0 / var0 + (double)N[a] / noise_var);
+        double mu_n = var_n * (mu0 / var0 + R[a] / noise_var);
+        double u1 = orc_rng_uniform(seed, seq, round, pos, ORC_RNG_BANDIT, (uint32_t)a, 0, 0);
+        double u2 = orc_rng_uniform(seed, seq, round, pos, ORC_RNG_BANDIT, (uint32_t)a, 0, 1);
+        double z = sqrt(-2.0 * log(1.0 - u1)) * cos(6.283185307179586476925 * u2);
+        val[a] = mu_n + sqrt(var_n) * z;
+        if (sample_out) sample_out[a] = val[a];
+    }
+    return argmax_first(val, A, tol, near_mask);
+}
+
+static int cmp_u32(const void* a, const void* b)
+{
+    uint32_t x = *(const uint32_t*)a, y = *(const uint32_t*)b;
+    return (x > y) - (x < y);
+}
+
+/* Beta(alpha, beta) with integer parameters, drawn exactly as an order
+ * statistic: the alpha-th smallest of alpha + beta - 1 i.i.d. uniforms is
+ * Beta(alpha, beta).  Uniform j is word j%4 of Philox draw j/4.  Returned as
+ * the 24-bit integer (value = result / 2^24). */
+uint32_t orc_beta_order_stat(uint32_t alpha, uint32_t beta,
+                             uint64_t seed, uint32_t seq, uint32_t round, uint32_t pos, uint32_t arm)
+{
+    uint32_t n = alpha + beta - 1;
+    uint32_t* u = (uint32_t*)malloc(sizeof(uint32_t) * (n + 4));
+    for (uint32_t j = 0; j < n; j += 4) {
+        uint32_t w[4];
+        orc_rng_words(seed, seq, round, pos, ORC_RNG_BANDIT, arm, j / 4, w);
+        for (int k = 0; k < 4; ++k) u[j + k] = w[k] >> 8;
+    }
+    qsort(u, n, sizeof(uint32_t), cmp_u32);
+    uint32_t r = u[alpha - 1];
+    free(u);
+    return r;
+}
+
+/* Thompson Sampling, Beta-Bernoulli (token level): theta_a ~ Beta(a0 + successes,
+ * b0 + failures); rewards are 0/1 so R[a] is an integer count. */
+int orc_ts_beta_select(const uint32_t* N, const double* R, int A, uint32_t a0, uint32_t b0,
+                       uint64_t seed, uint32_t seq, uint32_t round, uint32_t pos,
+                       uint32_t* sample_out)
+{
+    int best = 0;
+    uint32_t best_v = 0;
+    for (int a = 0; a < A; ++a) {
+        uint32_t succ = (uint32_t)R[a];
+        uint32_t fail = N[a] - succ;
+        uint32_t v = orc_beta_order_stat(a0 + succ, b0 + fail, seed, seq, round, pos, (uint32_t)a);
+        if (sample_out) sample_out[a] = v;
+        if (a == 0 || v > best_v) { best = a; best_v = v; }
+    }
+    return best;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Speculative-sampling verification of one sequence (Algorithm 1, verify    */
+/* and final-token steps; accept rule of the speculative-sampling papers).   */
+/* ------------------------------------------------------------------------- */
+typedef struct {
+    int accept_len;     /* |Y|                                              */
+    int next_token;     /* residual draw (rejection) or bonus draw          */
+    int next_lo, next_hi; /* draws at u -/+ tol                              */
+    int near_accept;    /* some |u_i - ratio_i| <= tol along the walk       */
+    int zero_residual;  /* residual mass was <= 0, drew from p instead      */
+    int bad_target;     /* a needed target row was invalid                  */
+    double ratio_at_stop; /* p/q at the rejected slot (or last accepted)     */
+} orc_verify_out;
+
+/* q_rows: the n draft rows (pointer to row 0, pos_stride elements apart);
+ * p_rows: n+1 target rows.  lse_q[i] = log-sum-exp of draft row i (scaled).
+ * scratch: 3*V doubles. */
+void orc_verify_sequence(const void* q_rows, long q_pos_stride, const void* p_rows, long p_pos_stride,
+                         int dtype, int V, float inv_Tq, float inv_Tp,
+                         const int32_t* x, int n, const double* lse_q,
+                         uint64_t seed, uint32_t seq, uint32_t round, double tol,
+                         double* scratch, orc_verify_out* out)
+{
+    size_t esz = (dtype == ORC_FP32) ? 4 : 2;
+    double* wp = scratch;
+    double* wq = scratch + V;
+    double* res = scratch + 2 * (size_t)V;
+    memset(out, 0, sizeof *out);
+    out->next_token = -1; out->next_lo = -1; out->next_hi = -1;
+
+    int a = n;
+    orc_rowstats sp;
+    for (int i = 0; i < n; ++i) {
+        const void* prow = (const char*)p_rows + (size_t)i * p_pos_stride * esz;
+        const void* qrow = (const char*)q_rows + (size_t)i * q_pos_stride * esz;
+        if (!orc_row_stats(prow, dtype, V, inv_Tp, wp, &sp)) { out->bad_target = 1; a = i; out->accept_len = a; return; }
+        double logp = load_logit(prow, dtype, x[i]) * (double)inv_Tp - sp.lse;
+        double logq = load_logit(qrow, dtype, x[i]) * (double)inv_Tq - lse_q[i];
+        double ratio = exp(logp - logq);                 /* p_i(x_i) / q_i(x_i)      */
+        double u = orc_rng_uniform(seed, seq, round, (uint32_t)i, ORC_RNG_ACCEPT, 0, 0, 0);
+        out->ratio_at_stop = ratio;
+        if (fabs(u - ratio) <= tol) out->near_accept = 1;
+        if (!(u < ratio)) { a = i; break; }              /* accept iff u < min(1, p/q) */
+    }
+    out->accept_len = a;
+
+    double u2 = orc_rng_uniform(seed, seq, round, (uint32_t)a, ORC_RNG_RESAMPLE, 0, 0, 0);
+    const void* prow = (const char*)p_rows + (size_t)a * p_pos_stride * esz;
+    if (a == n) {
+        /* every draft token accepted: bonus token from the next target row */
+        if (!orc_row_stats(prow, dtype, V, inv_Tp, wp, &sp)) { out->bad_target = 1; return; }
+        out->next_token = orc_sample_cdf(wp, V, sp.W, u2, tol, &out->next_lo, &out->next_hi);
+        return;
+    }
+    /* rejection at slot a: draw from norm(max(0, p - q)) of that slot.
+     * wp and sp still hold the rejected slot's target row. */
+    const void* qrow = (const char*)q_rows + (size_t)a * q_pos_stride * esz;
+    orc_rowstats sq;
+    orc_row_stats(qrow, dtype, V, inv_Tq, wq, &sq);
+    double Z = 0.0;
+    for (int v = 0; v < V; ++v) {
+        double r = wp[v] / sp.W - wq[v] / sq.W;
+        res[v] = r > 0.0 ? r : 0.0;
+        Z += res[v];
+    }
+    if (Z > 0.0) {
+        out->next_token = orc_sample_cdf(res, V, Z, u2, tol, &out->next_lo, &out->next_hi);
+    } else {
+        out->zero_residual = 1;
+        out->next_token = orc_sample_cdf(wp, V, sp.W, u2, tol, &out->next_lo, &out->next_hi);
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* The round engine: Algorithm 1 over a batch of independent sequences.      */
+/* ------------------------------------------------------------------------- */
+typedef struct {
+    int S, V, K, A, policy, level;
+    int P;                       /* bandits per sequence: 1 (sequence level) or K (token level) */
+    int rule_of_arm[ORC_MAX_ARMS];
+    /* parameters */
+    uint64_t seed;
+    int dtype;
+    float inv_Tq, inv_Tp;
+    orc_ruleparams rp;
+    double reward_alpha;         /* 0.5 */
+    int reward_kind;             /* 0 = r_blend, 1 = r_simple */
+    double ucb_c2;               /* 2 */
+    double ts_mu0, ts_var0, ts_noise_var;
+    uint32_t ts_beta_a0, ts_beta_b0;
+    double ada_lambda0, ada_acc0;
+    int token_update_all;        /* 1: every drafted position gets r_i = [i <= a]; 0: only i <= a+1 */
+    double tol;                  /* near-threshold band, 1e-6 */
+    /* per-sequence global ids (RNG stream of local sequence s is seq_id[s]) */
+    uint32_t* seq_id;
+    /* bandit statistics [S][P][A] */
+    uint32_t* cnt;
+    double* rsum;
+    double* rsum2;
+    /* AdaEDL state [S] */
+    double* lambda;
+    double* acc_rate;
+    /* round state */
+    uint32_t round;
+    int pos;
+    int drafted_any;
+    int verified;
+    int32_t* arm;                /* [S][K] arm index chosen per position (sequence level: same in all) */
+    int32_t* n_drafted;          /* [S] */
+    uint8_t* active;             /* [S] */
+    uint8_t* void_round;         /* [S] 1: first draft row invalid, nothing drafted */
+    double* sqrtH_prev;          /* [S] */
+    double* lse_q;               /* [S][K] */
+    double* feat;                /* [S][K][6]: m, lse, p1, p2, H, argmax */
+    int32_t* accept_len;         /* [S] */
+    double* reward;              /* [S] last sequence-level reward */
+    uint64_t status;
+    uint64_t rows_read;
+} orc_t;
+
+orc_t* orc_create(int S, int V, int K, int A, int policy, int level)
+{
+    if (S <= 0 || V <= 0 || K <= 0 || A <= 0 || A > ORC_MAX_ARMS) return NULL;
+    orc_t* h = (orc_t*)calloc(1, sizeof(orc_t));
+    h->S = S; h->V = V; h->K = K; h->A = A; h->policy = policy; h->level = level;
+    h->P = (level == ORC_TOKEN) ? K : 1;
+    for (int a = 0; a < A; ++a) h->rule_of_arm[a] = a % 5;   /* Table 1 order */
+    h->seed = 0; h->dtype = ORC_BF16; h->inv_Tq = 1.0f; h->inv_Tp = 1.0f;
+    h->rp.h_maxconf = 0.8; h->rp.h_svip = 0.6; h->rp.h_diff = 0.2; h->rp.h_margin = 0.2;
+    /* AdaEDL constants are not given in the paper; these are this build's choices. */
+    h->rp.ada_gamma = 0.2; h->rp.ada_alpha = 0.9; h->rp.ada_beta1 = 0.5; h->rp.ada_beta2 = 0.9; h->rp.ada_eps = 0.01;
+    h->ada_lambda0 = 0.4; h->ada_acc0 = 1.0;
+    h->reward_alpha = 0.5; h->reward_kind = 0; h->ucb_c2 = 2.0;
+    h->ts_mu0 = 0.0; h->ts_var0 = 1.0; h->ts_noise_var = 1.0;
+    h->ts_beta_a0 = 1; h->ts_beta_b0 = 1;
+    h->token_update_all = 1;
+    h->tol = 1e-6;
+    size_t spa = (size_t)S * h->P * A;
+    h->seq_id = (uint32_t*)calloc(S, sizeof(uint32_t));
+    for (int s = 0; s < S; ++s) h->seq_id[s] = (uint32_t)s;
+    h->cnt = (uint32_t*)calloc(spa, sizeof(uint32_t));
+    h->rsum = (double*)calloc(spa, sizeof(double));
+    h->rsum2 = (double*)calloc(spa, sizeof(double));
+    h->lambda = (double*)calloc(S, sizeof(double));
+    h->acc_rate = (double*)calloc(S, sizeof(double));
+    for (int s = 0; s < S; ++s) { h->lambda[s] = h->ada_lambda0; h->acc_rate[s] = h->ada_acc0; }
+    h->arm = (int32_t*)calloc((size_t)S * K, sizeof(int32_t));
+    h->n_drafted = (int32_t*)calloc(S, sizeof(int32_t));
+    h->active = (uint8_t*)calloc(S, 1);
+    h->void_round = (uint8_t*)calloc(S, 1);
+    h->sqrtH_prev = (double*)calloc(S, sizeof(double));
+    h->lse_q = (double*)calloc((size_t)S * K, sizeof(double));
+    h->feat = (double*)calloc((size_t)S * K * 6, sizeof(double));
+    h->accept_len = (int32_t*)calloc(S, sizeof(int32_t));
+    h->reward = (double*)calloc(S, sizeof(double));
+    return h;
+}
+
+void orc_destroy(orc_t* h)
+{
+    if (!h) return;
+    free(h->seq_id); free(h->cnt); free(h->rsum); free(h->rsum2); free(h->lambda); free(h->acc_rate);
+    free(h->arm); free(h->n_drafted); free(h->active); free(h->void_round); free(h->sqrtH_prev);
+    free(h->lse_q); free(h->feat); free(h->accept_len); free(h->reward);
+    free(h);
+}
+
+/* re-apply lambda0 / acc0 after the caller changed them (before round 0) */
+void orc_reset_adaedl(orc_t* h)
+{
+    for (int s = 0; s < h->S; ++s) { h->lambda[s] = h->ada_lambda0; h->acc_rate[s] = h->ada_acc0; }
+}
+
+static int select_arm(orc_t* h, int s, int slot, uint32_t pos, uint32_t* near_mask)
+{
+    size_t o = ((size_t)s * h->P + slot) * h->A;
+    const uint32_t* N = h->cnt + o;
+    const double* R = h->rsum + o;
+    uint32_t dummy;
+    if (!near_mask) near_mask = &dummy;
+    if (h->policy == ORC_UCB1) return orc_ucb1_select(N, R, h->A, h->ucb_c2, h->tol, NULL, near_mask);
+    if (h->policy == ORC_UCB_TUNED) return orc_ucb_tuned_select(N, R, h->rsum2 + o, h->A, h->tol, NULL, near_mask);
+    if (h->level == ORC_SEQ)
+        return orc_ts_gauss_select(N, R, h->A, h->ts_mu0, h->ts_var0, h->ts_noise_var,
+                                   h->seed, h->seq_id[s], h->round, pos, h->tol, NULL, near_mask);
+    int a = orc_ts_beta_select(N, R, h->A, h->ts_beta_a0, h->ts_beta_b0, h->seed, h->seq_id[s], h->round, pos, NULL);
+    *near_mask = 1u << a;     /* integer samples: exact on any machine */
+    return a;
+}
+
+/* One draft position for the whole batch (Algorithm 1, the loop body).
+ * logits: row of sequence s at logits + s * row_stride elements.
+ * Optional outputs (may be NULL): tok_lo/tok_hi = draws at u -/+ tol;
+ * near_rule[s] = rule quantity within tol of its threshold;
+ * arm_mask[s] = arms whose bandit value is within tol of the chosen one's. */
+int orc_draft_step(orc_t* h, const void* logits, long row_stride,
+                   int32_t* out_token, uint8_t* out_continue,
+                   int32_t* tok_lo, int32_t* tok_hi, uint8_t* near_rule, uint32_t* arm_mask)
+{
+    if (h->pos >= h->K || h->verified) return -2;
+    int i = h->pos;                       /* 0-based draft position */
+    size_t esz = (h->dtype == ORC_FP32) ? 4 : 2;
+    if (i == 0) {
+        for (int s = 0; s < h->S; ++s) { h->active[s] = 1; h->n_drafted[s] = 0; h->void_round[s] = 0; h->sqrtH_prev[s] = 0.0; }
+    }
+    uint64_t status = 0, rows = 0;
+    #pragma omp parallel for schedule(dynamic, 1) reduction(|:status) reduction(+:rows)
+    for (int s = 0; s < h->S; ++s) {
+        if (tok_lo) tok_lo[s] = -1;
+        if (tok_hi) tok_hi[s] = -1;
+        if (near_rule) near_rule[s] = 0;
+        if (arm_mask) arm_mask[s] = 0;
+        if (!h->active[s]) { out_token[s] = -1; out_continue[s] = 0; continue; }
+
+        /* which rule is consulted at this position */
+        int arm;
+        uint32_t mk = 0;
+        if (h->level == ORC_SEQ) {
+            if (i == 0) { arm = select_arm(h, s, 0, 0, &mk); for (int k = 0; k < h->K; ++k) h->arm[(size_t)s * h->K + k] = arm; }
+            else arm = h->arm[(size_t)s * h->K];
+        } else {
+            arm = select_arm(h, s, i, (uint32_t)i, &mk);
+            h->arm[(size_t)s * h->K + i] = arm;
+        }
+        if (arm_mask) arm_mask[s] = mk;
+
+        const void* row = (const char*)logits + (size_t)s * row_stride * esz;
+        double* w = (double*)malloc(sizeof(double) * h->V);
+        orc_rowstats st;
+        rows += 1;
+        if (!orc_row_stats(row, h->dtype, h->V, h->inv_Tq, w, &st)) {
+            /* unusable row: nothing is drafted at this position, the sequence stops */
+            status |= ORC_ST_BAD_DRAFT_ROW;
+            out_token[s] = -1; out_continue[s] = 0; h->active[s] = 0;
+            if (i == 0) h->void_round[s] = 1;
+            free(w);
+            continue;
+        }
+        double* f = h->feat + ((size_t)s * h->K + i) * 6;
+        f[0] = st.m; f[1] = st.lse; f[2] = st.p1; f[3] = st.p2; f[4] = st.H; f[5] = (double)st.argmax;
+        h->lse_q[(size_t)s * h->K + i] = st.lse;
+
+        /* x_i ~ M_q */
+        double u = orc_rng_uniform(h->seed, h->seq_id[s], h->round, (uint32_t)i, ORC_RNG_DRAFT, 0, 0, 0);
+        int lo, hi;
+        out_token[s] = orc_sample_cdf(w, h->V, st.W, u, h->tol, &lo, &hi);
+        if (tok_lo) tok_lo[s] = lo;
+        if (tok_hi) tok_hi[s] = hi;
+        free(w);
+        h->n_drafted[s] = i + 1;
+
+        /* does pi_theta signal stop at step i */
+        int near = 0;
+        int stop = orc_rule_stop(h->rule_of_arm[arm], st.p1, st.p2, st.H, h->sqrtH_prev[s], i > 0,
+                                 h->lambda[s], &h->rp, h->tol, &near);
+        h->sqrtH_prev[s] = sqrt(st.H);
+        if (i == h->K - 1) { stop = 1; near = 0; }      /* the loop ends at gamma */
+        if (near_rule) near_rule[s] = (uint8_t)near;
+        out_continue[s] = (uint8_t)!stop;
+        h->active[s] = (uint8_t)!stop;
+    }
+    h->status |= status;
+    h->rows_read += rows;
+    h->pos = i + 1;
+    h->drafted_any = 1;
+    return 0;
+}
+
+/* Verify + final token for the whole batch.  draft_logits [S][K][V] with the
+ * given strides (elements), target_logits [S][K+1][V], draft_tokens [S][K]. */
+int orc_verify(orc_t* h, const void* draft_logits, long q_seq_stride, long q_pos_stride,
+               const void* target_logits, long p_seq_stride, long p_pos_stride,
+               const int32_t* draft_tokens, int32_t* out_accept_len, int32_t* out_next_token,
+               int32_t* next_lo, int32_t* next_hi, uint8_t* near_accept)
+{
+    if (!h->drafted_any || h->verified) return -2;
+    size_t esz = (h->dtype == ORC_FP32) ? 4 : 2;
+    uint64_t status = 0, rows = 0;
+    #pragma omp parallel for schedule(dynamic, 1) reduction(|:status) reduction(+:rows)
+    for (int s = 0; s < h->S; ++s) {
+        double* scratch = (double*)malloc(sizeof(double) * 3 * (size_t)h->V);
+        orc_verify_out vo;
+        int n = h->n_drafted[s];
+        orc_verify_sequence((const char*)draft_logits + (size_t)s * q_seq_stride * esz, q_pos_stride,
+                            (const char*)target_logits + (size_t)s * p_seq_stride * esz, p_pos_stride,
+                            h->dtype, h->V, h->inv_Tq, h->inv_Tp,
+                            draft_tokens + (size_t)s * h->K, n, h->lse_q + (size_t)s * h->K,
+                            h->seed, h->seq_id[s], h->round, h->tol, scratch, &vo);
+        free(scratch);
+        if (vo.bad_target) status |= ORC_ST_BAD_TARGET_ROW;
+        if (vo.zero_residual) status |= ORC_ST_ZERO_RESIDUAL;
+        rows += (uint64_t)vo.accept_len + 1 + (vo.accept_len < n ? 1 : 0);
+        h->accept_len[s] = vo.accept_len;
+        out_accept_len[s] = vo.accept_len;
+        out_next_token[s] = vo.next_token;
+        if (next_lo) next_lo[s] = vo.next_lo;
+        if (next_hi) next_hi[s] = vo.next_hi;
+        if (near_accept) near_accept[s] = (uint8_t)vo.near_accept;
+    }
+    h->status |= status;
+    h->rows_read += rows;
+    h->verified = 1;
+    return 0;
+}
+
+/* update(pi_theta, |Y|, |X|, gamma): reward, arm statistics, AdaEDL state. */
+int orc_update(orc_t* h)
+{
+    if (!h->verified) return -2;
+    for (int s = 0; s < h->S; ++s) {
+        int n = h->n_drafted[s], a = h->accept_len[s];
+        h->reward[s] = 0.0;
+        if (n <= 0) continue;                      /* nothing drafted: no feedback */
+        if (h->level == ORC_SEQ) {
+            double r = h->reward_kind ? orc_reward_simple(a, h->K) : orc_reward_blend(a, n, h->K, h->reward_alpha);
+            size_t o = (size_t)s * h->A + h->arm[(size_t)s * h->K];
+            h->cnt[o] += 1; h->rsum[o] += r; h->rsum2[o] += r * r;
+            h->reward[s] = r;
+        } else {
+            int last = h->token_update_all ? n : (a + 1 < n ? a + 1 : n);
+            for (int i = 0; i < last; ++i) {
+                double r = (i < a) ? 1.0 : 0.0;    /* token i accepted or not */
+                size_t o = ((size_t)s * h->K + i) * h->A + h->arm[(size_t)s * h->K + i];
+                h->cnt[o] += 1; h->rsum[o] += r; h->rsum2[o] += r * r;
+            }
+            h->reward[s] = (double)a;
+        }
+        orc_adaedl_update(&h->lambda[s], &h->acc_rate[s], a, n, &h->rp);
+    }
+    h->round += 1; h->pos = 0; h->drafted_any = 0; h->verified = 0;
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Field access for the Python wrapper (pointers into the engine's arrays).  */
+/* ------------------------------------------------------------------------- */
+#define FIELD_PTR(name) void* orc_ptr_##name(orc_t* h) { return (void*)h->name; }
+FIELD_PTR(seq_id) FIELD_PTR(cnt) FIELD_PTR(rsum) FIELD_PTR(rsum2) FIELD_PTR(lambda) FIELD_PTR(acc_rate)
+FIELD_PTR(arm) FIELD_PTR(n_drafted) FIELD_PTR(active) FIELD_PTR(void_round) FIELD_PTR(sqrtH_prev)
+FIELD_PTR(lse_q) FIELD_PTR(feat) FIELD_PTR(accept_len) FIELD_PTR(reward) FIELD_PTR(rule_of_arm)
+
+int orc_get_P(orc_t* h) { return h->P; }
+uint32_t orc_get_round(orc_t* h) { return h->round; }
+int orc_get_pos(orc_t* h) { return h->pos; }
+uint64_t orc_get_status(orc_t* h) { return h->status; }
+uint64_t orc_get_rows(orc_t* h) { return h->rows_read; }
+
+/* parameter keys (the oracle's own numbering) */
+int orc_set_param(orc_t* h, const char* key, double v)
+{
+#define K_(s) (strcmp(key, s) == 0)
+    if (K_("seed")) h->seed = (uint64_t)v;
+    else if (K_("dtype")) h->dtype = (int)v;
+    else if (K_("inv_temp_draft")) h->inv_Tq = (float)v;
+    else if (K_("inv_temp_target")) h->inv_Tp = (float)v;
+    else if (K_("h_maxconf")) h->rp.h_maxconf = v;
+    else if (K_("h_svip")) h->rp.h_svip = v;
+    else if (K_("h_diff")) h->rp.h_diff = v;
+    else if (K_("h_margin")) h->rp.h_margin = v;
+    else if (K_("ada_gamma")) h->rp.ada_gamma = v;
+    else if (K_("ada_alpha")) h->rp.ada_alpha = v;
+    else if (K_("ada_beta1")) h->rp.ada_beta1 = v;
+    else if (K_("ada_beta2")) h->rp.ada_beta2 = v;
+    else if (K_("ada_eps")) h->rp.ada_eps = v;
+    else if (K_("ada_lambda0")) { h->ada_lambda0 = v; orc_reset_adaedl(h); }
+    else if (K_("ada_acc0")) { h->ada_acc0 = v; orc_reset_adaedl(h); }
+    else if (K_("reward_alpha")) h->reward_alpha = v;
+    else if (K_("reward_kind")) h->reward_kind = (int)v;
+    else if (K_("ucb_c2")) h->ucb_c2 = v;
+    else if (K_("ts_mu0")) h->ts_mu0 = v;
+    else if (K_("ts_var0")) h->ts_var0 = v;
+    else if (K_("ts_noise_var")) h->ts_noise_var = v;
+    else if (K_("ts_beta_a0")) h->ts_beta_a0 = (uint32_t)v;
+    else if (K_("ts_beta_b0")) h->ts_beta_b0 = (uint32_t)v;
+    else if (K_("token_update_all")) h->token_update_all = (int)v;
+    else if (K_("tol")) h->tol = v;
+    else return -1;
+#undef K_
+    return 0;
+}
+
+/* seed needs all 64 bits, which a double cannot carry */
+void orc_set_seed(orc_t* h, uint64_t seed) { h->seed = seed; }

@@ -1,0 +1,329 @@
+"""Pins for the oracle's verification step and round engine: speculative-sampling
+identities, distributional exactness on tiny vocabularies, Algorithm 1 invariants,
+and a hand re-derivation of whole rounds from the primitives."""
+import math
+
+import numpy as np
+import pytest
+import scipy.special as sps
+import scipy.stats as sst
+
+from oracle import oracle as orc
+
+
+def _logits_from_probs(p):
+    with np.errstate(divide="ignore"):
+        return np.log(np.asarray(p, dtype=np.float64)).astype(np.float32)
+
+
+def _softmax32(z):
+    return sps.softmax(z.astype(np.float64))
+
+
+# ------------------------------------------------------- verify, one sequence
+def test_p_equals_q_always_accepts():
+    rng = np.random.default_rng(0)
+    V, n = 50, 6
+    rows = rng.normal(size=(n + 1, V)).astype(np.float32) * 2
+    lse = [orc.row_stats(rows[i]).lse for i in range(n)]
+    for seq in range(200):
+        x = rng.integers(0, V, n)
+        out = orc.verify_sequence(rows[:n], rows, x, lse, seed=1, seq=seq, rnd=0)
+        assert out.accept_len == n                      # ratio == 1 > u always
+        assert 0 <= out.next_token < V                  # bonus token from row n
+
+
+def test_disjoint_support_always_rejects_and_residual_is_p():
+    V = 8
+    p = np.array([0.1, 0.2, 0.3, 0.4, 0, 0, 0, 0.0])
+    q = np.array([0, 0, 0, 0, 0.25, 0.25, 0.25, 0.25])
+    P = np.tile(_logits_from_probs(p), (3, 1))
+    Q = np.tile(_logits_from_probs(q), (2, 1))
+    lse = [orc.row_stats(Q[i]).lse for i in range(2)]
+    cnt = np.zeros(V)
+    n = 40000
+    for seq in range(n):
+        out = orc.verify_sequence(Q, P, [4 + seq % 4, 5], lse, seed=2, seq=seq, rnd=3)
+        assert out.accept_len == 0
+        assert not out.zero_residual
+        cnt[out.next_token] += 1
+    assert cnt[4:].sum() == 0
+    assert sst.chisquare(cnt[:4], n * p[:4]).pvalue > 1e-4
+
+
+def test_acceptance_frequency_is_sum_min_p_q():
+    rng = np.random.default_rng(1)
+    V = 10
+    zp = rng.normal(size=V).astype(np.float32) * 1.5
+    zq = (zp + rng.normal(size=V) * 0.8).astype(np.float32)
+    p, q = _softmax32(zp), _softmax32(zq)
+    P = np.stack([zp, zp])
+    Q = zq[None, :]
+    st, w = orc.row_stats(zq, want_w=True)
+    n, acc = 60000, 0
+    for seq in range(n):
+        u = orc.rng_uniform(4, seq, 0, 0, orc.RNG_DRAFT)
+        x = orc.sample_cdf(w, st.W, u)[0]
+        acc += orc.verify_sequence(Q, P, [x], [st.lse], seed=4, seq=seq, rnd=0).accept_len
+    beta = np.minimum(p, q).sum()
+    assert acc / n == pytest.approx(beta, abs=4 * math.sqrt(beta * (1 - beta) / n))
+
+
+def test_identical_rows_never_reach_the_residual():
+    # p == q: ratio is exactly 1, u < 1, so the walk cannot be rejected and the zero-mass
+    # residual (which only rounding could produce) is never consulted.
+    V = 6
+    z = np.linspace(-1, 1, V).astype(np.float32)
+    out = orc.verify_sequence(z[None, :], np.stack([z, z]), [2], [orc.row_stats(z).lse], seed=0, seq=0, rnd=0)
+    assert out.accept_len == 1 and not out.zero_residual
+
+
+def test_temperatures_enter_the_ratio():
+    V = 7
+    rng = np.random.default_rng(3)
+    zp = rng.normal(size=V).astype(np.float32)
+    zq = rng.normal(size=V).astype(np.float32)
+    tq, tp = np.float32(1.0), np.float32(1 / 0.7)
+    x = 3
+    lse_q = orc.row_stats(zq, inv_T=tq).lse
+    out = orc.verify_sequence(zq[None, :], np.stack([zp, zp]), [x], [lse_q], seed=0, seq=0, rnd=0,
+                              inv_Tq=tq, inv_Tp=tp)
+    p = sps.softmax(zp.astype(np.float64) * float(tp))
+    q = sps.softmax(zq.astype(np.float64) * float(tq))
+    assert out.ratio_at_stop == pytest.approx(p[x] / q[x], rel=1e-12)
+    u = orc.rng_uniform(0, 0, 0, 0, orc.RNG_ACCEPT)
+    assert out.accept_len == int(u < p[x] / q[x])
+
+
+# ------------------------------------------------------------- whole engine
+def _tiny_engine(S, V, K, A=5, policy=orc.UCB1, level=orc.SEQ, seed=0, **kw):
+    return orc.Oracle(S, V, K, A, policy, level, seed=seed, dtype=orc.FP32, **kw)
+
+
+def test_first_emitted_token_is_distributed_as_target():
+    # Speculative sampling is exact: whatever the draft distribution and the stop rule, the first token
+    # the round emits (x_1 if accepted, else the residual draw) follows p_1.
+    rng = np.random.default_rng(5)
+    V, K, S = 9, 3, 50000
+    zp = (rng.normal(size=(K + 1, V)) * 1.5).astype(np.float32)
+    zq = (zp[:K] + rng.normal(size=(K, V)) * 1.0).astype(np.float32)
+    D = np.ascontiguousarray(np.broadcast_to(zq, (S, K, V)))
+    T = np.ascontiguousarray(np.broadcast_to(zp, (S, K + 1, V)))
+    for policy, level, kw in ((orc.UCB1, orc.SEQ, {}), (orc.TS, orc.TOKEN, {}),
+                              (orc.UCB1, orc.SEQ, dict(A=2, arms=[orc.RULE_STATIC, orc.RULE_SVIPDIFF]))):
+        eng = _tiny_engine(S, V, K, policy=policy, level=level, seed=77, **kw)
+        toks = np.full((S, K), -1, np.int32)
+        for i in range(K):
+            r = eng.draft_step(D[:, i, :])
+            toks[:, i] = r["token"]
+        v = eng.verify(D, T, toks)
+        first = np.where(v["accept_len"] >= 1, toks[:, 0], v["next_token"])
+        cnt = np.bincount(first, minlength=V)
+        assert sst.chisquare(cnt, S * _softmax32(zp[0])).pvalue > 1e-4
+        # and the second emitted token, given that the first was accepted, follows p_2
+        n = eng.view("n_drafted")
+        sel = (v["accept_len"] >= 1) & (n >= 2)
+        second = np.where(v["accept_len"][sel] >= 2, toks[sel, 1], v["next_token"][sel])
+        sel2 = (v["accept_len"][sel] >= 2) | (v["accept_len"][sel] == 1)
+        cnt2 = np.bincount(second[sel2], minlength=V)
+        if kw:
+            assert cnt2.sum() > S // 10
+        if cnt2.sum() > 1000:
+            assert sst.chisquare(cnt2, cnt2.sum() * _softmax32(zp[1])).pvalue > 1e-4
+        eng.update()
+
+
+def test_invariants_over_rounds():
+    rng = np.random.default_rng(6)
+    S, V, K, A, rounds = 24, 40, 5, 5, 30
+    for policy, level in ((orc.UCB1, orc.SEQ), (orc.TS, orc.SEQ), (orc.UCB1, orc.TOKEN), (orc.TS, orc.TOKEN),
+                          (orc.UCB_TUNED, orc.SEQ)):
+        eng = _tiny_engine(S, V, K, A, policy, level, seed=9)
+        visits = np.zeros((S, K), np.int64)
+        for rnd in range(rounds):
+            scale = rng.choice([0.5, 3.0, 8.0])               # flat and peaked rows so all rules fire
+            T = (rng.normal(size=(S, K + 1, V)) * scale).astype(np.float32)
+            D = (T[:, :K] + rng.normal(size=(S, K, V)) * 0.7).astype(np.float32)
+            toks = np.full((S, K), -1, np.int32)
+            alive = np.ones(S, bool)
+            for i in range(K):
+                r = eng.draft_step(D[:, i, :])
+                assert np.all(r["token"][~alive] == -1) and np.all(r["cont"][~alive] == 0)
+                assert np.all((r["token"][alive] >= 0) & (r["token"][alive] < V))
+                toks[:, i] = r["token"]
+                alive &= r["cont"].astype(bool)
+            assert not alive.any()                            # forced stop at K
+            n = eng.view("n_drafted").copy()
+            assert np.all((1 <= n) & (n <= K))
+            assert np.all((toks >= 0).sum(axis=1) == n)
+            v = eng.verify(D, T, toks)
+            a = v["accept_len"]
+            assert np.all((0 <= a) & (a <= n))
+            assert np.all((v["next_token"] >= 0) & (v["next_token"] < V))
+            arms = eng.view("arm").copy()
+            eng.update()
+            for s in range(S):
+                visits[s, : n[s]] += 1
+            cnt, rs = eng.view("cnt"), eng.view("rsum")
+            assert np.all(rs >= 0) and np.all(rs <= cnt + 1e-12)
+            if level == orc.SEQ:
+                assert np.all(cnt.sum(axis=(1, 2)) == rnd + 1)
+                want = 0.5 * a / K + 0.5 * a / n
+                np.testing.assert_allclose(eng.view("reward"), want, rtol=1e-15)
+                if policy != orc.TS and rnd < A:
+                    assert np.all(arms[:, 0] == rnd)          # unplayed arms first, in order
+            else:
+                np.testing.assert_array_equal(cnt.sum(axis=2), visits)
+        assert eng.round == rounds
+
+
+def test_forced_stop_and_static_arm():
+    S, V, K = 4, 16, 6
+    eng = _tiny_engine(S, V, K, A=1, seed=1, arms=[orc.RULE_STATIC])
+    z = np.zeros((S, K, V), np.float32)
+    for i in range(K):
+        r = eng.draft_step(z[:, i, :])
+        assert np.all(r["cont"] == (0 if i == K - 1 else 1))
+    assert np.all(eng.view("n_drafted") == K)
+    with pytest.raises(RuntimeError):
+        eng.draft_step(z[:, 0, :])                            # a (K+1)-th step is a call-order error
+    eng2 = _tiny_engine(S, V, K)
+    with pytest.raises(RuntimeError):
+        eng2.update()
+
+
+def test_invalid_rows():
+    S, V, K = 3, 12, 4
+    eng = _tiny_engine(S, V, K, A=1, seed=1, arms=[orc.RULE_STATIC])
+    rng = np.random.default_rng(0)
+    D = rng.normal(size=(S, K, V)).astype(np.float32)
+    T = rng.normal(size=(S, K + 1, V)).astype(np.float32)
+    D[0, 0, 3] = np.nan            # sequence 0: nothing can be drafted this round
+    D[1, 2, :] = -np.inf           # sequence 1: stops after two tokens
+    toks = np.full((S, K), -1, np.int32)
+    for i in range(K):
+        toks[:, i] = eng.draft_step(D[:, i, :])["token"]
+    assert list(eng.view("n_drafted")) == [0, 2, K]
+    assert toks[0, 0] == -1 and toks[1, 2] == -1 and eng.status & orc.ST_BAD_DRAFT_ROW
+    v = eng.verify(D, T, toks)
+    assert v["accept_len"][0] == 0 and 0 <= v["next_token"][0] < V     # token from p_1
+    before = eng.view("cnt").copy()
+    eng.update()
+    after = eng.view("cnt")
+    assert after[0].sum() == before[0].sum()                  # no feedback without a draft
+    assert after[1].sum() == before[1].sum() + 1
+
+
+def test_round_rederived_from_primitives():
+    """Recomputes whole rounds in Python from the primitive functions (and numpy), checking the engine's
+    wiring: counters (seq id, round, position, purpose), which row feeds which step, state carried over."""
+    rng = np.random.default_rng(11)
+    S, V, K, A = 6, 30, 4, 5
+    seed = 123456789012345
+    ids = np.array([5, 17, 3, 1000, 42, 7], np.uint32)
+    eng = _tiny_engine(S, V, K, A, seed=seed, seq_ids=ids)
+    N = np.zeros((S, A), np.uint32)
+    R = np.zeros((S, A))
+    lam = np.full(S, 0.4)
+    for rnd in range(12):
+        T = (rng.normal(size=(S, K + 1, V)) * rng.choice([1.0, 6.0])).astype(np.float32)
+        D = (T[:, :K] + rng.normal(size=(S, K, V)) * 0.5).astype(np.float32)
+        toks = np.full((S, K), -1, np.int32)
+        got_tok, got_cont = [], []
+        for i in range(K):
+            r = eng.draft_step(D[:, i, :])
+            got_tok.append(r["token"])
+            got_cont.append(r["cont"])
+            toks[:, i] = r["token"]
+        v = eng.verify(D, T, toks)
+        eng.update()
+        for s in range(S):
+            sid = int(ids[s])
+            arm = orc.ucb1_select(N[s], R[s])[0]
+            prev, n = 0.0, 0
+            lse_q = []
+            for i in range(K):
+                st, w = orc.row_stats(D[s, i], want_w=True)
+                lse_q.append(st.lse)
+                u = orc.rng_uniform(seed, sid, rnd, i, orc.RNG_DRAFT)
+                x = orc.sample_cdf(w, st.W, u)[0]
+                assert got_tok[i][s] == x
+                stop = orc.rule_stop(arm, st.p1, st.p2, st.H, prev, int(i > 0), lam[s])[0] or i == K - 1
+                prev = math.sqrt(st.H)
+                assert got_cont[i][s] == (0 if stop else 1)
+                n = i + 1
+                if stop:
+                    break
+            for i in range(n, K):
+                assert got_tok[i][s] == -1 and got_cont[i][s] == 0
+            out = orc.verify_sequence(D[s], T[s], toks[s, :n], lse_q, seed, sid, rnd)
+            assert v["accept_len"][s] == out.accept_len and v["next_token"][s] == out.next_token
+            a = out.accept_len
+            # the walk itself, by hand
+            aa = n
+            for i in range(n):
+                p = sps.softmax(T[s, i].astype(np.float64))
+                q = sps.softmax(D[s, i].astype(np.float64))
+                u = orc.rng_uniform(seed, sid, rnd, i, orc.RNG_ACCEPT)
+                if not (u < p[toks[s, i]] / q[toks[s, i]]):
+                    aa = i
+                    break
+            assert aa == a
+            u2 = orc.rng_uniform(seed, sid, rnd, a, orc.RNG_RESAMPLE)
+            p = sps.softmax(T[s, a].astype(np.float64))
+            if a < n:
+                q = sps.softmax(D[s, a].astype(np.float64))
+                res = np.maximum(p - q, 0)
+                c = np.cumsum(res)
+                j = int(np.searchsorted(c, u2 * c[-1], side="right"))
+            else:
+                c = np.cumsum(p)
+                j = int(np.searchsorted(c, u2 * c[-1], side="right"))
+            if v["next_lo"][s] == v["next_hi"][s]:          # away from a CDF boundary the answer is unique
+                assert j == v["next_token"][s]
+            N[s, arm] += 1
+            R[s, arm] += orc.reward_blend(a, n, K)
+            lam[s] = orc.adaedl_update(lam[s], 1.0, a, n)[0]
+        np.testing.assert_array_equal(eng.view("cnt")[:, 0, :], N)
+        np.testing.assert_allclose(eng.view("rsum")[:, 0, :], R, rtol=1e-15)
+        np.testing.assert_allclose(eng.view("lambda"), lam, rtol=1e-15)
+
+
+def test_token_level_bandit_wiring():
+    rng = np.random.default_rng(12)
+    S, V, K, A = 5, 20, 4, 5
+    seed = 31
+    eng = _tiny_engine(S, V, K, A, policy=orc.TS, level=orc.TOKEN, seed=seed)
+    N = np.zeros((S, K, A), np.uint32)
+    R = np.zeros((S, K, A))
+    for rnd in range(15):
+        T = (rng.normal(size=(S, K + 1, V)) * 5).astype(np.float32)
+        D = (T[:, :K] + rng.normal(size=(S, K, V)) * 0.5).astype(np.float32)
+        toks = np.full((S, K), -1, np.int32)
+        for i in range(K):
+            toks[:, i] = eng.draft_step(D[:, i, :])["token"]
+        arms = eng.view("arm").copy()
+        n = eng.view("n_drafted").copy()
+        a = eng.verify(D, T, toks)["accept_len"]
+        eng.update()
+        for s in range(S):
+            for i in range(n[s]):
+                want = orc.ts_beta_select(N[s, i], R[s, i], seed, s, rnd, i)[0]
+                assert arms[s, i] == want
+            for i in range(n[s]):
+                N[s, i, arms[s, i]] += 1
+                R[s, i, arms[s, i]] += 1.0 if i < a[s] else 0.0
+        np.testing.assert_array_equal(eng.view("cnt"), N)
+        np.testing.assert_array_equal(eng.view("rsum"), R)
+
+
+def test_reward_kind_simple_and_token_update_switch():
+    S, V, K = 2, 10, 4
+    rng = np.random.default_rng(1)
+    T = (rng.normal(size=(S, K + 1, V)) * 4).astype(np.float32)
+    D = T[:, :K].copy()
+    eng = _tiny_engine(S, V, K, A=1, seed=2, arms=[orc.RULE_STATIC], reward_kind=1)
+    toks = np.stack([eng.draft_step(D[:, i, :])["token"] for i in range(K)], axis=1)
+    a = eng.verify(D, T, toks)["accept_len"]
+    eng.update()
+    np.testing.assert_allclose(eng.view("reward"), a / K)     # r_simple = |Y| / gamma
