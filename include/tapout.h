@@ -1,0 +1,257 @@
+/*
+ * libtapout: the batched, vocabulary-wide hot path of TapOut (arXiv 2511.02017),
+ * a bandit controller for dynamic speculative decoding, as CUDA kernels for
+ * NVIDIA B200 (sm_100a) behind a plain C ABI.
+ *
+ * One speculation round (the paper's Algorithm 1, everything except the two
+ * model forwards, whose logits the caller supplies):
+ *
+ *     for i in 0 .. k_max-1:   tapout_draft_step(h, draft_logits_i, tok, cont)
+ *     tapout_verify(h, draft_logits, target_logits, draft_tokens, acc_len, next_tok)
+ *     tapout_update(h)
+ *
+ * Conventions
+ *   - Every function returns TAPOUT_OK (0) or a negative tapout_error; nothing
+ *     throws across this boundary.  tapout_strerror() names a code.
+ *   - "device pointer" = memory of the CUDA device that was current when the
+ *     handle was created; "host pointer" = ordinary host memory.
+ *   - All device work is enqueued on the handle's stream (default: the legacy
+ *     default stream, settable with tapout_set_stream).  draft_step / verify /
+ *     update never synchronise the host.
+ *   - The caller owns every logits, token and output buffer.  The library owns
+ *     its bandit state and scratch memory, allocated in tapout_create and
+ *     released in tapout_destroy.
+ *   - Logit rows: base pointers 16-byte aligned and row strides a multiple of
+ *     16 bytes, otherwise TAPOUT_E_ALIGNMENT.  vocab itself may be any size.
+ *     -inf logits are legal (probability zero).  A row containing NaN or +inf,
+ *     or with no finite entry, is unusable: it sets a status bit, yields token
+ *     -1 and stops the sequence (see tapout_get_status).
+ *   - Randomness: Philox4x32-10 with key = seed and counter =
+ *     (global sequence id, round, position, purpose | arm << 4 | draw << 8);
+ *     purposes 0 draft sample, 1 acceptance test, 2 residual/bonus sample,
+ *     3 bandit.  A uniform is (word >> 8) * 2^-24.
+ */
+#ifndef TAPOUT_H
+#define TAPOUT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tapout tapout_t;
+
+typedef enum {
+    TAPOUT_OK = 0,
+    TAPOUT_E_INVALID_ARG = -1,  /* null pointer, size or enum out of range              */
+    TAPOUT_E_BAD_STATE = -2,    /* call order: e.g. verify before any draft step        */
+    TAPOUT_E_ALIGNMENT = -3,    /* a logits pointer or stride is not 16-byte aligned    */
+    TAPOUT_E_CUDA = -4,         /* a CUDA runtime call failed (tapout_last_cuda_error)  */
+    TAPOUT_E_ALLOC = -5,        /* out of host or device memory                         */
+    TAPOUT_E_UNSUPPORTED = -6   /* valid request this build does not implement          */
+} tapout_error;
+
+/* Bandit algorithm (Section 3.3) and action granularity (Section 3.1). */
+enum { TAPOUT_POLICY_UCB1 = 0, TAPOUT_POLICY_TS = 1, TAPOUT_POLICY_UCB_TUNED = 2 };
+enum { TAPOUT_LEVEL_SEQ = 0, TAPOUT_LEVEL_TOKEN = 1 };
+enum { TAPOUT_DTYPE_FP32 = 0, TAPOUT_DTYPE_BF16 = 1 };
+
+/* Stop rules: Table 1 in table order, plus a fixed-length arm that never stops early. */
+enum {
+    TAPOUT_RULE_MAXCONF = 0,   /* stop iff p(top-1) < h                       (h = 0.8)  */
+    TAPOUT_RULE_SVIP = 1,      /* stop iff sqrt(H) > h                        (h = 0.6)  */
+    TAPOUT_RULE_ADAEDL = 2,    /* stop iff 1 - sqrt(gamma*H) < lambda_t                  */
+    TAPOUT_RULE_SVIPDIFF = 3,  /* stop iff sqrt(H_t) - sqrt(H_{t-1}) > h      (h = 0.2)  */
+    TAPOUT_RULE_MARGIN = 4,    /* stop iff p(top-1) - p(top-2) < h            (h = 0.2)  */
+    TAPOUT_RULE_STATIC = 5     /* never stops before k_max                                */
+};
+
+/* Parameter keys for tapout_set_param_f64 / _i64 (legal only between rounds). */
+typedef enum {
+    TAPOUT_P_SEED = 0,             /* i64: Philox key (default 0)                                    */
+    TAPOUT_P_DTYPE = 1,            /* i64: TAPOUT_DTYPE_* of every logits tensor (default BF16)      */
+    TAPOUT_P_SEQ_OFFSET = 2,       /* i64: global id of local sequence 0 (sharding; default 0)       */
+    TAPOUT_P_INV_TEMP_DRAFT = 3,   /* f64: logits are multiplied by this (held as float; default 1)  */
+    TAPOUT_P_INV_TEMP_TARGET = 4,  /* f64: same for target logits                                    */
+    TAPOUT_P_STEP_ROW_STRIDE = 5,  /* i64: elements between rows of the draft_step input (default vocab) */
+    TAPOUT_P_Q_SEQ_STRIDE = 6,     /* i64: verify, draft tensor: elements between sequences (default k_max*vocab) */
+    TAPOUT_P_Q_POS_STRIDE = 7,     /* i64:   ... between positions (default vocab)                   */
+    TAPOUT_P_P_SEQ_STRIDE = 8,     /* i64: verify, target tensor: between sequences (default (k_max+1)*vocab) */
+    TAPOUT_P_P_POS_STRIDE = 9,     /* i64:   ... between positions (default vocab)                   */
+    TAPOUT_P_H_MAXCONF = 10,       /* f64: Table 1 thresholds                                        */
+    TAPOUT_P_H_SVIP = 11,
+    TAPOUT_P_H_DIFF = 12,
+    TAPOUT_P_H_MARGIN = 13,
+    TAPOUT_P_ADA_GAMMA = 14,       /* f64: AdaEDL's own gamma, alpha, beta1, beta2, epsilon          */
+    TAPOUT_P_ADA_ALPHA = 15,
+    TAPOUT_P_ADA_BETA1 = 16,
+    TAPOUT_P_ADA_BETA2 = 17,
+    TAPOUT_P_ADA_EPS = 18,
+    TAPOUT_P_ADA_LAMBDA0 = 19,     /* f64: initial lambda; setting it re-initialises every sequence  */
+    TAPOUT_P_ADA_ACC0 = 20,        /* f64: initial accept_rate; likewise                             */
+    TAPOUT_P_REWARD_ALPHA = 21,    /* f64: alpha of r_blend (default 0.5)                            */
+    TAPOUT_P_REWARD_KIND = 22,     /* i64: 0 = r_blend, 1 = r_simple                                 */
+    TAPOUT_P_UCB_C2 = 23,          /* f64: the 2 in sqrt(2 ln t / N)                                 */
+    TAPOUT_P_TS_MU0 = 24,          /* f64: Gaussian-TS prior mean, prior variance, noise variance    */
+    TAPOUT_P_TS_VAR0 = 25,
+    TAPOUT_P_TS_NOISE_VAR = 26,
+    TAPOUT_P_TS_BETA_A0 = 27,      /* i64: Beta-TS prior (integers; default 1, 1)                    */
+    TAPOUT_P_TS_BETA_B0 = 28,
+    TAPOUT_P_TOKEN_UPDATE_ALL = 29,/* i64: 1 = every drafted position gets r_i = [i accepted] (default); 0 = only up to the first rejection */
+    TAPOUT_P_ROW_SEGMENTS = 30,    /* i64: CTAs that share one draft row (0 = chosen from n_seq)     */
+    TAPOUT_P_TOKEN_OUT_STRIDE = 31,/* i64: elements between sequences in out_token of draft_step (default 1); with k_max the
+                                      caller can aim step i at column i of its [n_seq][k_max] token matrix  */
+    TAPOUT_P_PROFILE = 32,         /* i64: 1 = time the two streaming kernels with CUDA events (tapout_get_profile) */
+    TAPOUT_P__COUNT = 33
+} tapout_param;
+
+/* Sticky status bits reported by tapout_get_status. */
+#define TAPOUT_ST_BAD_DRAFT_ROW 1ull   /* a draft row was unusable                              */
+#define TAPOUT_ST_BAD_TARGET_ROW 2ull  /* a target row was unusable                             */
+#define TAPOUT_ST_ZERO_RESIDUAL 4ull   /* max(0,p-q) summed to 0; the token was drawn from p    */
+#define TAPOUT_ST_BAD_TOKEN 8ull       /* a draft token passed to verify was outside [0, vocab) */
+
+const char* tapout_strerror(int code);
+
+/* Text of the last CUDA error seen by this handle ("" if none).  Owned by the handle. */
+const char* tapout_last_cuda_error(const tapout_t* h);
+
+/*
+ * Problem statement, Section 3.1.  Creates the controller for n_seq independent
+ * sequences: each has its own bandit over n_arms arms -- one bandit per sequence
+ * (TAPOUT_LEVEL_SEQ: the arm is chosen at the start of a drafting session) or
+ * one per (sequence, draft position) (TAPOUT_LEVEL_TOKEN).  Arm a applies rule
+ * a % 5 of Table 1 unless tapout_set_arms says otherwise.  k_max is the paper's
+ * maximum draft length gamma.  Allocates all state and scratch on the current
+ * device; statistics start at zero, round = 0.
+ *   1 <= n_seq, 2 <= vocab, 1 <= k_max <= 1024, 1 <= n_arms <= 16.
+ */
+int tapout_create(tapout_t** out, int n_seq, int vocab, int k_max, int n_arms, int policy, int level);
+
+/* Frees the handle and all device memory it owns (synchronises its stream first). */
+int tapout_destroy(tapout_t* h);
+
+/* stream: a cudaStream_t (as void*); the library neither creates nor destroys it. */
+int tapout_set_stream(tapout_t* h, void* stream);
+
+int tapout_set_param_f64(tapout_t* h, int key, double value);
+int tapout_set_param_i64(tapout_t* h, int key, int64_t value);
+int tapout_get_param_f64(const tapout_t* h, int key, double* value);
+int tapout_get_param_i64(const tapout_t* h, int key, int64_t* value);
+
+/* rule_ids: host pointer to n TAPOUT_RULE_* values, n == n_arms.  Between rounds only. */
+int tapout_set_arms(tapout_t* h, const int32_t* rule_ids, int n);
+
+/*
+ * Algorithm 1, loop body, for draft position i = number of draft steps already
+ * taken this round (at most k_max calls per round, else TAPOUT_E_BAD_STATE).
+ * For each sequence still drafting:
+ *   - softmax statistics of its row of draft_logits (Table 1 features: top-1 and
+ *     top-2 probability, entropy in nats; also max, log-sum-exp, argmax),
+ *   - x_i ~ softmax(row) by inverse CDF in token order with one Philox uniform,
+ *   - the stop rule of the bandit-selected arm (sequence level: arm chosen at
+ *     i = 0; token level: chosen here) -> out_continue.
+ * Sequences that already stopped: row not read, out_token = -1, out_continue = 0.
+ * At i = k_max-1 out_continue is 0 for all.
+ *   draft_logits : device, [n_seq] rows of vocab elements, TAPOUT_P_STEP_ROW_STRIDE apart
+ *   out_token    : device, int32 [n_seq] (TAPOUT_P_TOKEN_OUT_STRIDE elements apart)
+ *   out_continue : device, uint8 [n_seq], 1 = keep drafting
+ */
+int tapout_draft_step(tapout_t* h, const void* draft_logits, int32_t* out_token, uint8_t* out_continue);
+
+/*
+ * Algorithm 1, verification and final token, as speculative sampling: walking
+ * i = 0 .. n-1 (n = tokens drafted), token x_i is accepted iff
+ * u_i < min(1, p_i(x_i) / q_i(x_i)); the walk ends at the first rejection and
+ * target rows after it are not read.  out_accept_len = |Y|.  out_next_token is
+ * drawn from norm(max(0, p - q)) of the rejected slot, or from the target row
+ * n (the bonus token) when everything was accepted.
+ *   draft_probs   : device, the draft LOGITS tensor [n_seq][k_max][vocab] whose rows
+ *                   were given to tapout_draft_step this round (strides
+ *                   TAPOUT_P_Q_*); q is re-derived from them with the saved
+ *                   log-sum-exp of each row
+ *   target_logits : device, [n_seq][k_max+1][vocab] (strides TAPOUT_P_P_*)
+ *   draft_tokens  : device, int32 [n_seq][k_max]; entries at positions >= n are ignored
+ *   out_accept_len, out_next_token : device, int32 [n_seq]
+ * TAPOUT_E_BAD_STATE if no draft step ran this round or verify already ran.
+ */
+int tapout_verify(tapout_t* h, const void* draft_probs, const void* target_logits,
+                  const int32_t* draft_tokens, int32_t* out_accept_len, int32_t* out_next_token);
+
+/*
+ * Algorithm 1, update(pi, |Y|, |X|, gamma): Section 3.2 rewards (sequence level
+ * r_blend = alpha |Y|/gamma + (1-alpha) |Y|/|X|; token level 1 per accepted
+ * token, 0 otherwise), N_a += 1, R_a += r for the arm(s) played, the AdaEDL
+ * lambda / accept_rate update (Appendix A.1), then round += 1.
+ * TAPOUT_E_BAD_STATE unless tapout_verify ran this round.
+ */
+int tapout_update(tapout_t* h);
+
+/*
+ * One whole round from HOST memory: copies the round's logits to the device,
+ * runs k_max draft steps, verify and update, and copies the results back.
+ * Blocks until done.  Host arrays: draft_logits [n_seq][k_max][vocab],
+ * target_logits [n_seq][k_max+1][vocab] (contiguous), out_draft_tokens
+ * int32 [n_seq][k_max] (-1 beyond the drafted length), out_accept_len and
+ * out_next_token int32 [n_seq].  Device staging buffers are allocated on first use.
+ */
+int tapout_round_host(tapout_t* h, const void* draft_logits, const void* target_logits,
+                      int32_t* out_draft_tokens, int32_t* out_accept_len, int32_t* out_next_token);
+
+/*
+ * Table 1 features of arbitrary rows, outside any round (kernel-level checks and
+ * timing of the row pass): out_features, device float [n_rows][6] = max of the
+ * scaled logits, log-sum-exp, top-1 probability, top-2 probability, entropy
+ * (nats), argmax.  logits: device, n_rows <= n_seq rows, row_stride elements
+ * apart, dtype TAPOUT_P_DTYPE, scaled by inv_temp.  Uses the handle's scratch;
+ * legal only between rounds.  Unusable rows give NaN features and argmax -1.
+ */
+int tapout_row_stats(tapout_t* h, const void* logits, int n_rows, int64_t row_stride, double inv_temp,
+                     float* out_features);
+
+/*
+ * State: bandit statistics, AdaEDL state and the current round's bookkeeping in
+ * one blob (checkpoint/resume, arm-value read-out, test resynchronisation).
+ * Fields, each a dense C array: "cnt" u32 [S][P][A], "rsum" f64 [S][P][A],
+ * "rsum2" f64 [S][P][A], "lambda" f64 [S], "acc_rate" f64 [S], "arm" i32 [S][K],
+ * "n_drafted" i32 [S], "active" i32 [S], "sqrtH_prev" f64 [S], "lse_q" f64 [S][K],
+ * "feat" f32 [S][K][6], "accept_len" i32 [S], "reward" f64 [S]
+ * (S = n_seq, K = k_max, A = n_arms, P = 1 or K by level).
+ * get/set take HOST pointers to tapout_state_bytes() bytes and synchronise the stream.
+ */
+int tapout_state_bytes(const tapout_t* h, size_t* bytes);
+int tapout_state_field(const tapout_t* h, const char* name, size_t* offset, size_t* bytes);
+int tapout_get_state(tapout_t* h, void* host_dst);
+int tapout_set_state(tapout_t* h, const void* host_src);
+
+/* round = completed rounds; pos = draft steps taken in the current round. */
+int tapout_get_round(const tapout_t* h, uint32_t* round, int32_t* pos);
+
+/* Resume: sets the number of completed rounds (it is part of every Philox counter).  Between rounds only. */
+int tapout_set_round(tapout_t* h, uint32_t round);
+
+/*
+ * Synchronises the stream and reports the sticky status bits and the running
+ * counts of logit rows the method needed: draft rows, target rows, and draft
+ * rows re-read for a residual.  Any pointer may be NULL.
+ */
+int tapout_get_status(tapout_t* h, uint64_t* bits, uint64_t* rows_draft, uint64_t* rows_target,
+                      uint64_t* rows_residual);
+
+/*
+ * With TAPOUT_P_PROFILE = 1 every launch of the two streaming kernels (0: draft row pass,
+ * 1: verification walk) is bracketed by CUDA events on the handle's stream.  Synchronises,
+ * returns the summed device time in milliseconds and the number of launches since the last
+ * reset; reset != 0 clears both.
+ */
+int tapout_get_profile(tapout_t* h, int kernel, double* ms, uint64_t* launches, int reset);
+
+/* Kernels launched by this handle so far (host-side count). */
+int tapout_get_launch_count(const tapout_t* h, uint64_t* launches);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TAPOUT_H */

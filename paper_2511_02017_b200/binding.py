@@ -1,0 +1,248 @@
+"""Thin ctypes binding over libtapout.so: same names as the C ABI (include/tapout.h),
+argument marshalling only.  torch is used for device memory and streams; every step of the
+method runs in the library's CUDA kernels.  There is no CPU fallback: if the library cannot be
+loaded, `load()` raises.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libtapout.so")
+
+OK, E_INVALID_ARG, E_BAD_STATE, E_ALIGNMENT, E_CUDA, E_ALLOC, E_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
+POLICY_UCB1, POLICY_TS, POLICY_UCB_TUNED = 0, 1, 2
+LEVEL_SEQ, LEVEL_TOKEN = 0, 1
+DTYPE_FP32, DTYPE_BF16 = 0, 1
+RULE_MAXCONF, RULE_SVIP, RULE_ADAEDL, RULE_SVIPDIFF, RULE_MARGIN, RULE_STATIC = range(6)
+ST_BAD_DRAFT_ROW, ST_BAD_TARGET_ROW, ST_ZERO_RESIDUAL, ST_BAD_TOKEN = 1, 2, 4, 8
+
+# parameter keys, in the order of tapout_param
+_PARAM_NAMES = [
+    "seed", "dtype", "seq_offset", "inv_temp_draft", "inv_temp_target", "step_row_stride", "q_seq_stride",
+    "q_pos_stride", "p_seq_stride", "p_pos_stride", "h_maxconf", "h_svip", "h_diff", "h_margin", "ada_gamma",
+    "ada_alpha", "ada_beta1", "ada_beta2", "ada_eps", "ada_lambda0", "ada_acc0", "reward_alpha", "reward_kind",
+    "ucb_c2", "ts_mu0", "ts_var0", "ts_noise_var", "ts_beta_a0", "ts_beta_b0", "token_update_all", "row_segments",
+    "token_out_stride", "profile",
+]
+PARAM = {n: i for i, n in enumerate(_PARAM_NAMES)}
+_INT_PARAMS = {"seed", "dtype", "seq_offset", "step_row_stride", "q_seq_stride", "q_pos_stride", "p_seq_stride",
+               "p_pos_stride", "reward_kind", "ts_beta_a0", "ts_beta_b0", "token_update_all", "row_segments",
+               "token_out_stride", "profile"}
+
+EXPORTS = [
+    "tapout_strerror", "tapout_last_cuda_error", "tapout_create", "tapout_destroy", "tapout_set_stream",
+    "tapout_set_param_f64", "tapout_set_param_i64", "tapout_get_param_f64", "tapout_get_param_i64",
+    "tapout_set_arms", "tapout_draft_step", "tapout_verify", "tapout_update", "tapout_round_host",
+    "tapout_row_stats", "tapout_state_bytes", "tapout_state_field", "tapout_get_state", "tapout_set_state",
+    "tapout_get_round", "tapout_set_round", "tapout_get_status", "tapout_get_profile", "tapout_get_launch_count",
+]
+
+_STATE_FIELDS = {
+    "cnt": (np.uint32, "SPA"), "rsum": (np.float64, "SPA"), "rsum2": (np.float64, "SPA"),
+    "lambda": (np.float64, "S"), "acc_rate": (np.float64, "S"), "arm": (np.int32, "SK"),
+    "n_drafted": (np.int32, "S"), "active": (np.int32, "S"), "sqrtH_prev": (np.float64, "S"),
+    "lse_q": (np.float64, "SK"), "feat": (np.float32, "SK6"), "accept_len": (np.int32, "S"),
+    "reward": (np.float64, "S"),
+}
+
+_lib = None
+
+
+class TapoutError(RuntimeError):
+    def __init__(self, code, where, detail=""):
+        self.code = code
+        msg = "%s: %s (%d)" % (where, load().tapout_strerror(code).decode(), code)
+        if detail:
+            msg += " [" + detail + "]"
+        super().__init__(msg)
+
+
+def load():
+    """Loads libtapout.so (built in-tree by paper_2511_02017_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError("libtapout.so is not built: run `python -m paper_2511_02017_b200.build` "
+                          "(expected at %s); there is no fallback path" % LIB_PATH)
+    L = C.CDLL(LIB_PATH)
+    vp, i32, i64, dbl = C.c_void_p, C.c_int, C.c_int64, C.c_double
+    L.tapout_strerror.restype = C.c_char_p
+    L.tapout_strerror.argtypes = [i32]
+    L.tapout_last_cuda_error.restype = C.c_char_p
+    L.tapout_last_cuda_error.argtypes = [vp]
+    L.tapout_create.argtypes = [C.POINTER(vp), i32, i32, i32, i32, i32, i32]
+    L.tapout_destroy.argtypes = [vp]
+    L.tapout_set_stream.argtypes = [vp, vp]
+    L.tapout_set_param_f64.argtypes = [vp, i32, dbl]
+    L.tapout_set_param_i64.argtypes = [vp, i32, i64]
+    L.tapout_get_param_f64.argtypes = [vp, i32, C.POINTER(dbl)]
+    L.tapout_get_param_i64.argtypes = [vp, i32, C.POINTER(i64)]
+    L.tapout_set_arms.argtypes = [vp, vp, i32]
+    L.tapout_draft_step.argtypes = [vp, vp, vp, vp]
+    L.tapout_verify.argtypes = [vp, vp, vp, vp, vp, vp]
+    L.tapout_update.argtypes = [vp]
+    L.tapout_round_host.argtypes = [vp, vp, vp, vp, vp, vp]
+    L.tapout_row_stats.argtypes = [vp, vp, i32, i64, dbl, vp]
+    L.tapout_state_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
+    L.tapout_state_field.argtypes = [vp, C.c_char_p, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+    L.tapout_get_state.argtypes = [vp, vp]
+    L.tapout_set_state.argtypes = [vp, vp]
+    L.tapout_get_round.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(C.c_int32)]
+    L.tapout_set_round.argtypes = [vp, C.c_uint32]
+    L.tapout_get_status.argtypes = [vp] + [C.POINTER(C.c_uint64)] * 4
+    L.tapout_get_profile.argtypes = [vp, i32, C.POINTER(dbl), C.POINTER(C.c_uint64), i32]
+    L.tapout_get_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
+    for name in EXPORTS:
+        getattr(L, name)
+    _lib = L
+    return L
+
+
+def _dev_ptr(t, dtype=None):
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError("expected a CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError("expected dtype %s, got %s" % (dtype, t.dtype))
+    return C.c_void_p(t.data_ptr())
+
+
+class Tapout:
+    """One controller handle.  Method names follow the C ABI without the `tapout_` prefix."""
+
+    def __init__(self, n_seq, vocab, k_max, n_arms, policy, level, **params):
+        self.L = load()
+        self.S, self.V, self.K, self.A = n_seq, vocab, k_max, n_arms
+        self.P = k_max if level == LEVEL_TOKEN else 1
+        self.h = C.c_void_p()
+        rc = self.L.tapout_create(C.byref(self.h), n_seq, vocab, k_max, n_arms, policy, level)
+        if rc != OK:
+            self.h = None
+            raise TapoutError(rc, "tapout_create")
+        for k, v in params.items():
+            self.set_param(k, v)
+
+    def _check(self, rc, where):
+        if rc != OK:
+            detail = self.L.tapout_last_cuda_error(self.h).decode() if rc == E_CUDA else ""
+            raise TapoutError(rc, where, detail)
+
+    def destroy(self):
+        if getattr(self, "h", None):
+            self.L.tapout_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def set_stream(self, stream):
+        ptr = stream.cuda_stream if isinstance(stream, torch.cuda.Stream) else int(stream or 0)
+        self._check(self.L.tapout_set_stream(self.h, C.c_void_p(ptr)), "tapout_set_stream")
+
+    def set_param(self, name, value):
+        if name == "arms":
+            return self.set_arms(value)
+        key = PARAM[name]
+        if name in _INT_PARAMS:
+            v = int(value)
+            if name == "seed" and v >= 1 << 63:
+                v -= 1 << 64
+            self._check(self.L.tapout_set_param_i64(self.h, key, v), "tapout_set_param_i64(%s)" % name)
+        else:
+            self._check(self.L.tapout_set_param_f64(self.h, key, float(value)), "tapout_set_param_f64(%s)" % name)
+
+    def get_param(self, name):
+        key = PARAM[name]
+        if name in _INT_PARAMS:
+            v = C.c_int64()
+            self._check(self.L.tapout_get_param_i64(self.h, key, C.byref(v)), "tapout_get_param_i64")
+            return v.value
+        v = C.c_double()
+        self._check(self.L.tapout_get_param_f64(self.h, key, C.byref(v)), "tapout_get_param_f64")
+        return v.value
+
+    def set_arms(self, rule_ids):
+        a = np.ascontiguousarray(rule_ids, dtype=np.int32)
+        self._check(self.L.tapout_set_arms(self.h, a.ctypes.data_as(C.c_void_p), a.shape[0]), "tapout_set_arms")
+
+    def draft_step(self, draft_logits, out_token, out_continue):
+        self._check(self.L.tapout_draft_step(self.h, _dev_ptr(draft_logits), _dev_ptr(out_token, torch.int32),
+                                             _dev_ptr(out_continue, torch.uint8)), "tapout_draft_step")
+
+    def verify(self, draft_probs, target_logits, draft_tokens, out_accept_len, out_next_token):
+        self._check(self.L.tapout_verify(self.h, _dev_ptr(draft_probs), _dev_ptr(target_logits),
+                                         _dev_ptr(draft_tokens, torch.int32), _dev_ptr(out_accept_len, torch.int32),
+                                         _dev_ptr(out_next_token, torch.int32)), "tapout_verify")
+
+    def update(self):
+        self._check(self.L.tapout_update(self.h), "tapout_update")
+
+    def round_host(self, draft_logits, target_logits, out_draft_tokens, out_accept_len, out_next_token):
+        """All arguments are CPU tensors (pinned or not); blocks until the round is done."""
+        for t in (draft_logits, target_logits, out_draft_tokens, out_accept_len, out_next_token):
+            if t.is_cuda or not t.is_contiguous():
+                raise TypeError("round_host takes contiguous host tensors")
+        self._check(self.L.tapout_round_host(self.h, C.c_void_p(draft_logits.data_ptr()),
+                                             C.c_void_p(target_logits.data_ptr()),
+                                             C.c_void_p(out_draft_tokens.data_ptr()),
+                                             C.c_void_p(out_accept_len.data_ptr()),
+                                             C.c_void_p(out_next_token.data_ptr())), "tapout_round_host")
+
+    def row_stats(self, logits, n_rows, row_stride, inv_temp, out_features):
+        self._check(self.L.tapout_row_stats(self.h, _dev_ptr(logits), n_rows, row_stride, float(inv_temp),
+                                            _dev_ptr(out_features, torch.float32)), "tapout_row_stats")
+
+    # ---- state
+    def state_bytes(self):
+        n = C.c_size_t()
+        self._check(self.L.tapout_state_bytes(self.h, C.byref(n)), "tapout_state_bytes")
+        return n.value
+
+    def state_field(self, name):
+        off, nb = C.c_size_t(), C.c_size_t()
+        self._check(self.L.tapout_state_field(self.h, name.encode(), C.byref(off), C.byref(nb)), "tapout_state_field")
+        return off.value, nb.value
+
+    def get_state(self):
+        """Host copy of the state blob as a dict of numpy arrays that alias one buffer (key '_blob')."""
+        blob = np.zeros(self.state_bytes(), dtype=np.uint8)
+        self._check(self.L.tapout_get_state(self.h, blob.ctypes.data_as(C.c_void_p)), "tapout_get_state")
+        out = {"_blob": blob}
+        dims = {"S": (self.S,), "SK": (self.S, self.K), "SK6": (self.S, self.K, 6), "SPA": (self.S, self.P, self.A)}
+        for name, (dt, shp) in _STATE_FIELDS.items():
+            off, nb = self.state_field(name)
+            out[name] = blob[off:off + nb].view(dt).reshape(dims[shp])
+        return out
+
+    def set_state(self, state):
+        blob = state["_blob"]
+        self._check(self.L.tapout_set_state(self.h, blob.ctypes.data_as(C.c_void_p)), "tapout_set_state")
+
+    def get_round(self):
+        r, p = C.c_uint32(), C.c_int32()
+        self._check(self.L.tapout_get_round(self.h, C.byref(r), C.byref(p)), "tapout_get_round")
+        return r.value, p.value
+
+    def set_round(self, rnd):
+        self._check(self.L.tapout_set_round(self.h, int(rnd)), "tapout_set_round")
+
+    def get_status(self):
+        v = [C.c_uint64() for _ in range(4)]
+        self._check(self.L.tapout_get_status(self.h, *[C.byref(x) for x in v]), "tapout_get_status")
+        return dict(bits=v[0].value, rows_draft=v[1].value, rows_target=v[2].value, rows_residual=v[3].value)
+
+    def get_profile(self, kernel, reset=False):
+        ms, n = C.c_double(), C.c_uint64()
+        self._check(self.L.tapout_get_profile(self.h, kernel, C.byref(ms), C.byref(n), int(reset)), "tapout_get_profile")
+        return ms.value, n.value
+
+    def get_launch_count(self):
+        n = C.c_uint64()
+        self._check(self.L.tapout_get_launch_count(self.h, C.byref(n)), "tapout_get_launch_count")
+        return n.value

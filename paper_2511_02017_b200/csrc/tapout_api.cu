@@ -1,0 +1,597 @@
+// The C ABI of libtapout (see include/tapout.h): handle, argument checks, call-order state
+// machine, launches.  Host code only decides what to launch; every step of the method runs
+// in the kernels of tapout_kernels.cuh.
+#include "tapout.h"
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "tapout_kernels.cuh"
+
+using namespace tpo;
+
+namespace {
+
+struct Field { const char* name; size_t offset, bytes; };
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+struct tapout {
+    Params p{};
+    int device = 0;
+    int n_sm = 0;
+    cudaStream_t stream = nullptr;
+    uint64_t seed = 0;
+    int64_t step_stride = 0, q_seq = 0, q_pos = 0, p_seq = 0, p_pos = 0;
+    int nseg_user = 0;
+    // call-order state (host mirror; the device never has to be asked)
+    uint32_t round = 0;
+    int pos = 0;
+    bool verified = false;
+    // device memory
+    char* d_state = nullptr;
+    size_t state_bytes = 0;
+    std::vector<Field> fields;
+    State st{};
+    char* d_scratch = nullptr;
+    Scratch sc{};
+    int grid_rows = 0, grid_walk = 0;
+    // host-round staging
+    char* d_stage = nullptr;
+    size_t stage_bytes = 0;
+    uint64_t launches = 0;
+    std::string cuda_err;
+    int64_t tok_stride = 1;
+    // optional event timing of the two streaming kernels
+    bool profile = false;
+    std::vector<cudaEvent_t> ev[2];      // start/stop pairs not yet read back
+    double prof_ms[2] = {0.0, 0.0};
+    uint64_t prof_n[2] = {0, 0};
+};
+
+namespace {
+
+int fail_cuda(tapout* h, cudaError_t e, const char* what) {
+    h->cuda_err = std::string(what) + ": " + cudaGetErrorString(e);
+    return TAPOUT_E_CUDA;
+}
+
+#define TP_CUDA(h, call)                                   \
+    do {                                                   \
+        cudaError_t e__ = (call);                          \
+        if (e__ != cudaSuccess) return fail_cuda(h, e__, #call); \
+    } while (0)
+
+#define TP_LAUNCHED(h)                                     \
+    do {                                                   \
+        (h)->launches += 1;                                \
+        cudaError_t e__ = cudaPeekAtLastError();           \
+        if (e__ != cudaSuccess) return fail_cuda(h, e__, "kernel launch"); \
+    } while (0)
+
+int elem_bytes(const tapout* h) { return h->p.dtype == DT_BF16 ? 2 : 4; }
+int chunk_of(const tapout* h) { return h->p.dtype == DT_BF16 ? chunk_elems<DT_BF16>() : chunk_elems<DT_FP32>(); }
+
+bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
+bool stride_ok(const tapout* h, int64_t stride_elems) { return stride_elems > 0 && (stride_elems * elem_bytes(h)) % 16 == 0; }
+
+float c_of(float inv_T) { return (float)((double)inv_T * kLog2e); }
+
+// Scratch sizes depend on dtype (chunk length) and on the row split: (re)allocated when those change.
+int setup_scratch(tapout* h) {
+    Params& p = h->p;
+    const int CH = chunk_of(h);
+    p.NC = (p.V + CH - 1) / CH;
+    int nseg = h->nseg_user;
+    if (nseg <= 0) {
+        const long long want = 4LL * h->n_sm * 4;                 // about four waves of resident CTAs
+        nseg = (int)((want + p.S - 1) / p.S);
+        const int cap = p.NC / kWarps > 0 ? p.NC / kWarps : 1;    // keep every warp of a CTA busy
+        if (nseg > cap) nseg = cap;
+    }
+    if (nseg < 1) nseg = 1;
+    if (nseg > kMaxSeg) nseg = kMaxSeg;
+    if (nseg > p.NC) nseg = p.NC;
+    p.nseg = nseg;
+
+    if (h->d_scratch) { cudaFree(h->d_scratch); h->d_scratch = nullptr; }
+    size_t off = 0;
+    const size_t o_seg = off;    off = align_up(off + sizeof(SegRec) * (size_t)p.S * p.nseg, 256);
+    const size_t o_cdf = off;    off = align_up(off + sizeof(float2) * (size_t)p.S * p.NC, 256);
+    const size_t o_list = off;   off = align_up(off + sizeof(int32_t) * 2 * (size_t)p.S, 256);
+    const size_t o_count = off;  off = align_up(off + sizeof(int32_t) * 4, 256);
+    const size_t o_order = off;  off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
+    const size_t o_status = off; off = align_up(off + sizeof(unsigned long long) * 4, 256);
+    TP_CUDA(h, cudaMalloc(&h->d_scratch, off));
+    TP_CUDA(h, cudaMemsetAsync(h->d_scratch, 0, off, h->stream));
+    h->sc.seg = reinterpret_cast<SegRec*>(h->d_scratch + o_seg);
+    h->sc.cdf = reinterpret_cast<float2*>(h->d_scratch + o_cdf);
+    h->sc.list = reinterpret_cast<int32_t*>(h->d_scratch + o_list);
+    h->sc.count = reinterpret_cast<int32_t*>(h->d_scratch + o_count);
+    h->sc.order = reinterpret_cast<int32_t*>(h->d_scratch + o_order);
+    h->sc.status = reinterpret_cast<unsigned long long*>(h->d_scratch + o_status);
+
+    const long long items = (long long)p.S * p.nseg;
+    const long long res_rows = (long long)h->n_sm * 4;
+    h->grid_rows = (int)(items < res_rows ? items : res_rows);
+    const long long res_walk = (long long)h->n_sm * 3;
+    h->grid_walk = (int)(p.S < res_walk ? p.S : res_walk);
+    return TAPOUT_OK;
+}
+
+int reset_round_state(tapout* h, int reset_adaedl) {
+    const int blocks = (h->p.S + 255) / 256;
+    k_reset_round<<<blocks, 256, 0, h->stream>>>(h->p, h->st, h->sc, reset_adaedl);
+    TP_LAUNCHED(h);
+    return TAPOUT_OK;
+}
+
+bool between_rounds(const tapout* h) { return h->pos == 0 && !h->verified; }
+
+// Reads back and releases the pending event pairs of kernel k (synchronises on each stop event).
+int drain_profile(tapout* h, int k) {
+    for (size_t i = 0; i + 1 < h->ev[k].size(); i += 2) {
+        float ms = 0.f;
+        cudaError_t e = cudaEventSynchronize(h->ev[k][i + 1]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, h->ev[k][i], h->ev[k][i + 1]);
+        cudaEventDestroy(h->ev[k][i]);
+        cudaEventDestroy(h->ev[k][i + 1]);
+        if (e != cudaSuccess) { h->ev[k].clear(); return fail_cuda(h, e, "profile events"); }
+        h->prof_ms[k] += ms;
+        h->prof_n[k] += 1;
+    }
+    h->ev[k].clear();
+    return TAPOUT_OK;
+}
+
+int profile_mark(tapout* h, int k) {
+    if (!h->profile) return TAPOUT_OK;
+    if (h->ev[k].size() >= 8192 && h->ev[k].size() % 2 == 0) { int rc = drain_profile(h, k); if (rc) return rc; }
+    cudaEvent_t e;
+    TP_CUDA(h, cudaEventCreate(&e));
+    h->ev[k].push_back(e);
+    TP_CUDA(h, cudaEventRecord(e, h->stream));
+    return TAPOUT_OK;
+}
+
+int draft_step_impl(tapout* h, const void* logits, int64_t stride, int32_t* out_token, int64_t tok_stride,
+                    uint8_t* out_continue) {
+    if (!h || !logits || !out_token || !out_continue) return TAPOUT_E_INVALID_ARG;
+    if (h->verified || h->pos >= h->p.K) return TAPOUT_E_BAD_STATE;
+    if (!aligned16(logits) || !stride_ok(h, stride)) return TAPOUT_E_ALIGNMENT;
+    const int parity = h->pos & 1;
+    const float c = c_of(h->p.inv_Tq);
+    { int rc = profile_mark(h, 0); if (rc) return rc; }
+    if (h->p.dtype == DT_BF16)
+        k_draft_rows<DT_BF16><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->sc, logits, stride, parity, -1, c);
+    else
+        k_draft_rows<DT_FP32><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->sc, logits, stride, parity, -1, c);
+    TP_LAUNCHED(h);
+    { int rc = profile_mark(h, 0); if (rc) return rc; }
+    const int blocks = (h->p.S + 3) / 4;
+    if (h->p.dtype == DT_BF16)
+        k_draft_finish<DT_BF16><<<blocks, 128, 0, h->stream>>>(h->p, h->st, h->sc, logits, stride, h->pos, parity,
+                                                               h->round, c, out_token, tok_stride, out_continue);
+    else
+        k_draft_finish<DT_FP32><<<blocks, 128, 0, h->stream>>>(h->p, h->st, h->sc, logits, stride, h->pos, parity,
+                                                               h->round, c, out_token, tok_stride, out_continue);
+    TP_LAUNCHED(h);
+    h->pos += 1;
+    return TAPOUT_OK;
+}
+
+int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const void* pl, int64_t p_seq, int64_t p_pos,
+                const int32_t* toks, int32_t* out_acc, int32_t* out_next) {
+    if (!h || !q || !pl || !toks || !out_acc || !out_next) return TAPOUT_E_INVALID_ARG;
+    if (h->pos == 0 || h->verified) return TAPOUT_E_BAD_STATE;
+    if (!aligned16(q) || !aligned16(pl) || !stride_ok(h, q_seq) || !stride_ok(h, q_pos) || !stride_ok(h, p_seq) ||
+        !stride_ok(h, p_pos))
+        return TAPOUT_E_ALIGNMENT;
+    k_verify_prepare<<<1, 1024, 0, h->stream>>>(h->p, h->st, h->sc);
+    TP_LAUNCHED(h);
+    const size_t smem = sizeof(float2) * (size_t)h->p.NC;
+    const float cq = c_of(h->p.inv_Tq), cp = c_of(h->p.inv_Tp);
+    { int rc = profile_mark(h, 1); if (rc) return rc; }
+    if (h->p.dtype == DT_BF16)
+        k_verify_walk<DT_BF16><<<h->grid_walk, kThreads, smem, h->stream>>>(h->p, h->st, h->sc, q, q_seq, q_pos, pl, p_seq,
+                                                                          p_pos, toks, h->round, cq, cp, out_acc, out_next);
+    else
+        k_verify_walk<DT_FP32><<<h->grid_walk, kThreads, smem, h->stream>>>(h->p, h->st, h->sc, q, q_seq, q_pos, pl, p_seq,
+                                                                          p_pos, toks, h->round, cq, cp, out_acc, out_next);
+    TP_LAUNCHED(h);
+    { int rc = profile_mark(h, 1); if (rc) return rc; }
+    h->verified = true;
+    return TAPOUT_OK;
+}
+
+int update_impl(tapout* h) {
+    if (!h) return TAPOUT_E_INVALID_ARG;
+    if (!h->verified) return TAPOUT_E_BAD_STATE;
+    k_update<<<(h->p.S + 255) / 256, 256, 0, h->stream>>>(h->p, h->st, h->sc);
+    TP_LAUNCHED(h);
+    h->round += 1;
+    h->pos = 0;
+    h->verified = false;
+    return TAPOUT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* tapout_strerror(int code) {
+    switch (code) {
+    case TAPOUT_OK: return "ok";
+    case TAPOUT_E_INVALID_ARG: return "invalid argument";
+    case TAPOUT_E_BAD_STATE: return "call out of order for the current round";
+    case TAPOUT_E_ALIGNMENT: return "logits pointer or stride not 16-byte aligned";
+    case TAPOUT_E_CUDA: return "CUDA runtime error";
+    case TAPOUT_E_ALLOC: return "out of memory";
+    case TAPOUT_E_UNSUPPORTED: return "not supported";
+    default: return "unknown error";
+    }
+}
+
+const char* tapout_last_cuda_error(const tapout_t* h) { return h ? h->cuda_err.c_str() : ""; }
+
+int tapout_create(tapout_t** out, int n_seq, int vocab, int k_max, int n_arms, int policy, int level) {
+    if (!out) return TAPOUT_E_INVALID_ARG;
+    *out = nullptr;
+    if (n_seq < 1 || vocab < 2 || k_max < 1 || k_max > 1024 || n_arms < 1 || n_arms > kMaxArms) return TAPOUT_E_INVALID_ARG;
+    if (policy < 0 || policy > 2 || level < 0 || level > 1) return TAPOUT_E_INVALID_ARG;
+    if ((long long)n_seq * k_max * n_arms > (1LL << 28)) return TAPOUT_E_INVALID_ARG;
+    tapout* h = new (std::nothrow) tapout();
+    if (!h) return TAPOUT_E_ALLOC;
+    Params& p = h->p;
+    p.S = n_seq; p.V = vocab; p.K = k_max; p.A = n_arms; p.policy = policy; p.level = level;
+    p.P = (level == TAPOUT_LEVEL_TOKEN) ? k_max : 1;
+    p.dtype = DT_BF16;
+    for (int a = 0; a < kMaxArms; ++a) p.rule_of_arm[a] = a % 5;
+    p.seed_lo = p.seed_hi = 0; p.seq_offset = 0;
+    p.inv_Tq = p.inv_Tp = 1.0f;
+    p.h_maxconf = 0.8; p.h_svip = 0.6; p.h_diff = 0.2; p.h_margin = 0.2;
+    // AdaEDL constants: the paper lists the symbols without values; these are this library's defaults.
+    p.ada_gamma = 0.2; p.ada_alpha = 0.9; p.ada_beta1 = 0.5; p.ada_beta2 = 0.9; p.ada_eps = 0.01;
+    p.ada_lambda0 = 0.4; p.ada_acc0 = 1.0;
+    p.reward_alpha = 0.5; p.ucb_c2 = 2.0; p.ts_mu0 = 0.0; p.ts_var0 = 1.0; p.ts_noise_var = 1.0;
+    p.ts_a0 = 1; p.ts_b0 = 1; p.reward_kind = 0; p.token_update_all = 1;
+    h->step_stride = vocab;
+    h->q_seq = (int64_t)k_max * vocab; h->q_pos = vocab;
+    h->p_seq = (int64_t)(k_max + 1) * vocab; h->p_pos = vocab;
+
+    cudaError_t e = cudaGetDevice(&h->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->n_sm, cudaDevAttrMultiProcessorCount, h->device);
+    if (e != cudaSuccess) { delete h; return TAPOUT_E_CUDA; }
+
+    // state blob
+    const size_t S = n_seq, K = k_max, PA = (size_t)p.P * n_arms;
+    size_t off = 0;
+    auto add = [&](const char* name, size_t bytes) { h->fields.push_back({name, off, bytes}); off = align_up(off + bytes, 256); };
+    add("cnt", 4 * S * PA); add("rsum", 8 * S * PA); add("rsum2", 8 * S * PA);
+    add("lambda", 8 * S); add("acc_rate", 8 * S); add("arm", 4 * S * K); add("n_drafted", 4 * S);
+    add("active", 4 * S); add("sqrtH_prev", 8 * S); add("lse_q", 8 * S * K); add("feat", 4 * S * K * kFeat);
+    add("accept_len", 4 * S); add("reward", 8 * S);
+    h->state_bytes = off;
+    if (cudaMalloc(&h->d_state, off) != cudaSuccess) { delete h; return TAPOUT_E_ALLOC; }
+    cudaMemset(h->d_state, 0, off);
+    auto at = [&](int i) { return h->d_state + h->fields[i].offset; };
+    h->st.cnt = (uint32_t*)at(0); h->st.rsum = (double*)at(1); h->st.rsum2 = (double*)at(2);
+    h->st.lambda = (double*)at(3); h->st.acc_rate = (double*)at(4); h->st.arm = (int32_t*)at(5);
+    h->st.n_drafted = (int32_t*)at(6); h->st.active = (int32_t*)at(7); h->st.sqrtH_prev = (double*)at(8);
+    h->st.lse_q = (double*)at(9); h->st.feat = (float*)at(10); h->st.accept_len = (int32_t*)at(11);
+    h->st.reward = (double*)at(12);
+
+    int rc = setup_scratch(h);
+    if (rc == TAPOUT_OK) rc = reset_round_state(h, 1);
+    if (rc != TAPOUT_OK) { tapout_destroy(h); return rc == TAPOUT_E_CUDA ? TAPOUT_E_ALLOC : rc; }
+    *out = h;
+    return TAPOUT_OK;
+}
+
+int tapout_destroy(tapout_t* h) {
+    if (!h) return TAPOUT_E_INVALID_ARG;
+    cudaStreamSynchronize(h->stream);
+    for (int k = 0; k < 2; ++k) { for (cudaEvent_t e : h->ev[k]) cudaEventDestroy(e); h->ev[k].clear(); }
+    if (h->d_state) cudaFree(h->d_state);
+    if (h->d_scratch) cudaFree(h->d_scratch);
+    if (h->d_stage) cudaFree(h->d_stage);
+    delete h;
+    return TAPOUT_OK;
+}
+
+int tapout_set_stream(tapout_t* h, void* stream) {
+    if (!h) return TAPOUT_E_INVALID_ARG;
+    if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
+    TP_CUDA(h, cudaStreamSynchronize(h->stream));
+    h->stream = reinterpret_cast<cudaStream_t>(stream);
+    return TAPOUT_OK;
+}
+
+int tapout_set_param_i64(tapout_t* h, int key, int64_t v) {
+    if (!h) return TAPOUT_E_INVALID_ARG;
+    if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
+    Params& p = h->p;
+    switch (key) {
+    case TAPOUT_P_SEED: h->seed = (uint64_t)v; p.seed_lo = (uint32_t)h->seed; p.seed_hi = (uint32_t)(h->seed >> 32); return TAPOUT_OK;
+    case TAPOUT_P_DTYPE:
+        if (v != DT_FP32 && v != DT_BF16) return TAPOUT_E_INVALID_ARG;
+        if (p.dtype != (int)v) {
+            p.dtype = (int)v;
+            TP_CUDA(h, cudaStreamSynchronize(h->stream));
+            int rc = setup_scratch(h);
+            if (rc != TAPOUT_OK) return rc;
+            return reset_round_state(h, 0);
+        }
+        return TAPOUT_OK;
+    case TAPOUT_P_SEQ_OFFSET: if (v < 0 || v > 0xffffffffLL) return TAPOUT_E_INVALID_ARG; p.seq_offset = (uint32_t)v; return TAPOUT_OK;
+    case TAPOUT_P_STEP_ROW_STRIDE: if (v < p.V) return TAPOUT_E_INVALID_ARG; h->step_stride = v; return TAPOUT_OK;
+    case TAPOUT_P_Q_SEQ_STRIDE: if (v < p.V) return TAPOUT_E_INVALID_ARG; h->q_seq = v; return TAPOUT_OK;
+    case TAPOUT_P_Q_POS_STRIDE: if (v < p.V) return TAPOUT_E_INVALID_ARG; h->q_pos = v; return TAPOUT_OK;
+    case TAPOUT_P_P_SEQ_STRIDE: if (v < p.V) return TAPOUT_E_INVALID_ARG; h->p_seq = v; return TAPOUT_OK;
+    case TAPOUT_P_P_POS_STRIDE: if (v < p.V) return TAPOUT_E_INVALID_ARG; h->p_pos = v; return TAPOUT_OK;
+    case TAPOUT_P_REWARD_KIND: if (v != 0 && v != 1) return TAPOUT_E_INVALID_ARG; p.reward_kind = (int)v; return TAPOUT_OK;
+    case TAPOUT_P_TS_BETA_A0: if (v < 1 || v > (1 << 20)) return TAPOUT_E_INVALID_ARG; p.ts_a0 = (uint32_t)v; return TAPOUT_OK;
+    case TAPOUT_P_TS_BETA_B0: if (v < 1 || v > (1 << 20)) return TAPOUT_E_INVALID_ARG; p.ts_b0 = (uint32_t)v; return TAPOUT_OK;
+    case TAPOUT_P_TOKEN_UPDATE_ALL: p.token_update_all = v ? 1 : 0; return TAPOUT_OK;
+    case TAPOUT_P_TOKEN_OUT_STRIDE: if (v < 1) return TAPOUT_E_INVALID_ARG; h->tok_stride = v; return TAPOUT_OK;
+    case TAPOUT_P_PROFILE: h->profile = v != 0; return TAPOUT_OK;
+    case TAPOUT_P_ROW_SEGMENTS: {
+        if (v < 0 || v > kMaxSeg) return TAPOUT_E_INVALID_ARG;
+        h->nseg_user = (int)v;
+        TP_CUDA(h, cudaStreamSynchronize(h->stream));
+        int rc = setup_scratch(h);
+        if (rc != TAPOUT_OK) return rc;
+        return reset_round_state(h, 0);
+    }
+    default: return TAPOUT_E_INVALID_ARG;
+    }
+}
+
+int tapout_set_param_f64(tapout_t* h, int key, double v) {
+    if (!h) return TAPOUT_E_INVALID_ARG;
+    if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
+    if (v != v) return TAPOUT_E_INVALID_ARG;
+    Params& p = h->p;
+    switch (key) {
+    case TAPOUT_P_INV_TEMP_DRAFT: if (!(v > 0.0) || !((float)v < 1e30f)) return TAPOUT_E_INVALID_ARG; p.inv_Tq = (float)v; return TAPOUT_OK;
+    case TAPOUT_P_INV_TEMP_TARGET: if (!(v > 0.0) || !((float)v < 1e30f)) return TAPOUT_E_INVALID_ARG; p.inv_Tp = (float)v; return TAPOUT_OK;
+    case TAPOUT_P_H_MAXCONF: p.h_maxconf = v; return TAPOUT_OK;
+    case TAPOUT_P_H_SVIP: p.h_svip = v; return TAPOUT_OK;
+    case TAPOUT_P_H_DIFF: p.h_diff = v; return TAPOUT_OK;
+    case TAPOUT_P_H_MARGIN: p.h_margin = v; return TAPOUT_OK;
+    case TAPOUT_P_ADA_GAMMA: p.ada_gamma = v; return TAPOUT_OK;
+    case TAPOUT_P_ADA_ALPHA: p.ada_alpha = v; return TAPOUT_OK;
+    case TAPOUT_P_ADA_BETA1: p.ada_beta1 = v; return TAPOUT_OK;
+    case TAPOUT_P_ADA_BETA2: p.ada_beta2 = v; return TAPOUT_OK;
+    case TAPOUT_P_ADA_EPS: p.ada_eps = v; return TAPOUT_OK;
+    case TAPOUT_P_ADA_LAMBDA0: p.ada_lambda0 = v; return reset_round_state(h, 1);
+    case TAPOUT_P_ADA_ACC0: p.ada_acc0 = v; return reset_round_state(h, 1);
+    case TAPOUT_P_REWARD_ALPHA: p.reward_alpha = v; return TAPOUT_OK;
+    case TAPOUT_P_UCB_C2: if (v < 0.0) return TAPOUT_E_INVALID_ARG; p.ucb_c2 = v; return TAPOUT_OK;
+    case TAPOUT_P_TS_MU0: p.ts_mu0 = v; return TAPOUT_OK;
+    case TAPOUT_P_TS_VAR0: if (!(v > 0.0)) return TAPOUT_E_INVALID_ARG; p.ts_var0 = v; return TAPOUT_OK;
+    case TAPOUT_P_TS_NOISE_VAR: if (!(v > 0.0)) return TAPOUT_E_INVALID_ARG; p.ts_noise_var = v; return TAPOUT_OK;
+    default: return TAPOUT_E_INVALID_ARG;
+    }
+}
+
+int tapout_get_param_i64(const tapout_t* h, int key, int64_t* v) {
+    if (!h || !v) return TAPOUT_E_INVALID_ARG;
+    const Params& p = h->p;
+    switch (key) {
+    case TAPOUT_P_SEED: *v = (int64_t)h->seed; return TAPOUT_OK;
+    case TAPOUT_P_DTYPE: *v = p.dtype; return TAPOUT_OK;
+    case TAPOUT_P_SEQ_OFFSET: *v = p.seq_offset; return TAPOUT_OK;
+    case TAPOUT_P_STEP_ROW_STRIDE: *v = h->step_stride; return TAPOUT_OK;
+    case TAPOUT_P_Q_SEQ_STRIDE: *v = h->q_seq; return TAPOUT_OK;
+    case TAPOUT_P_Q_POS_STRIDE: *v = h->q_pos; return TAPOUT_OK;
+    case TAPOUT_P_P_SEQ_STRIDE: *v = h->p_seq; return TAPOUT_OK;
+    case TAPOUT_P_P_POS_STRIDE: *v = h->p_pos; return TAPOUT_OK;
+    case TAPOUT_P_REWARD_KIND: *v = p.reward_kind; return TAPOUT_OK;
+    case TAPOUT_P_TS_BETA_A0: *v = p.ts_a0; return TAPOUT_OK;
+    case TAPOUT_P_TS_BETA_B0: *v = p.ts_b0; return TAPOUT_OK;
+    case TAPOUT_P_TOKEN_UPDATE_ALL: *v = p.token_update_all; return TAPOUT_OK;
+    case TAPOUT_P_ROW_SEGMENTS: *v = p.nseg; return TAPOUT_OK;
+    case TAPOUT_P_TOKEN_OUT_STRIDE: *v = h->tok_stride; return TAPOUT_OK;
+    case TAPOUT_P_PROFILE: *v = h->profile ? 1 : 0; return TAPOUT_OK;
+    default: return TAPOUT_E_INVALID_ARG;
+    }
+}
+
+int tapout_get_param_f64(const tapout_t* h, int key, double* v) {
+    if (!h || !v) return TAPOUT_E_INVALID_ARG;
+    const Params& p = h->p;
+    switch (key) {
+    case TAPOUT_P_INV_TEMP_DRAFT: *v = p.inv_Tq; return TAPOUT_OK;
+    case TAPOUT_P_INV_TEMP_TARGET: *v = p.inv_Tp; return TAPOUT_OK;
+    case TAPOUT_P_H_MAXCONF: *v = p.h_maxconf; return TAPOUT_OK;
+    case TAPOUT_P_H_SVIP: *v = p.h_svip; return TAPOUT_OK;
+    case TAPOUT_P_H_DIFF: *v = p.h_diff; return TAPOUT_OK;
+    case TAPOUT_P_H_MARGIN: *v = p.h_margin; return TAPOUT_OK;
+    case TAPOUT_P_ADA_GAMMA: *v = p.ada_gamma; return TAPOUT_OK;
+    case TAPOUT_P_ADA_ALPHA: *v = p.ada_alpha; return TAPOUT_OK;
+    case TAPOUT_P_ADA_BETA1: *v = p.ada_beta1; return TAPOUT_OK;
+    case TAPOUT_P_ADA_BETA2: *v = p.ada_beta2; return TAPOUT_OK;
+    case TAPOUT_P_ADA_EPS: *v = p.ada_eps; return TAPOUT_OK;
+    case TAPOUT_P_ADA_LAMBDA0: *v = p.ada_lambda0; return TAPOUT_OK;
+    case TAPOUT_P_ADA_ACC0: *v = p.ada_acc0; return TAPOUT_OK;
+    case TAPOUT_P_REWARD_ALPHA: *v = p.reward_alpha; return TAPOUT_OK;
+    case TAPOUT_P_UCB_C2: *v = p.ucb_c2; return TAPOUT_OK;
+    case TAPOUT_P_TS_MU0: *v = p.ts_mu0; return TAPOUT_OK;
+    case TAPOUT_P_TS_VAR0: *v = p.ts_var0; return TAPOUT_OK;
+    case TAPOUT_P_TS_NOISE_VAR: *v = p.ts_noise_var; return TAPOUT_OK;
+    default: return TAPOUT_E_INVALID_ARG;
+    }
+}
+
+int tapout_set_arms(tapout_t* h, const int32_t* rule_ids, int n) {
+    if (!h || !rule_ids || n != h->p.A) return TAPOUT_E_INVALID_ARG;
+    if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
+    for (int a = 0; a < n; ++a)
+        if (rule_ids[a] < 0 || rule_ids[a] > TAPOUT_RULE_STATIC) return TAPOUT_E_INVALID_ARG;
+    for (int a = 0; a < n; ++a) h->p.rule_of_arm[a] = rule_ids[a];
+    return TAPOUT_OK;
+}
+
+int tapout_draft_step(tapout_t* h, const void* draft_logits, int32_t* out_token, uint8_t* out_continue) {
+    if (!h) return TAPOUT_E_INVALID_ARG;
+    return draft_step_impl(h, draft_logits, h->step_stride, out_token, h->tok_stride, out_continue);
+}
+
+int tapout_verify(tapout_t* h, const void* draft_probs, const void* target_logits, const int32_t* draft_tokens,
+                  int32_t* out_accept_len, int32_t* out_next_token) {
+    if (!h) return TAPOUT_E_INVALID_ARG;
+    return verify_impl(h, draft_probs, h->q_seq, h->q_pos, target_logits, h->p_seq, h->p_pos, draft_tokens,
+                       out_accept_len, out_next_token);
+}
+
+int tapout_update(tapout_t* h) { return update_impl(h); }
+
+int tapout_round_host(tapout_t* h, const void* draft_logits, const void* target_logits, int32_t* out_draft_tokens,
+                      int32_t* out_accept_len, int32_t* out_next_token) {
+    if (!h || !draft_logits || !target_logits || !out_draft_tokens || !out_accept_len || !out_next_token)
+        return TAPOUT_E_INVALID_ARG;
+    if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
+    const Params& p = h->p;
+    const size_t S = p.S, K = p.K, V = p.V, esz = elem_bytes(h);
+    if ((V * esz) % 16 != 0) return TAPOUT_E_ALIGNMENT;
+    const size_t qb = S * K * V * esz, pb = S * (K + 1) * V * esz;
+    size_t off = 0;
+    const size_t o_q = off;    off = align_up(off + qb, 256);
+    const size_t o_p = off;    off = align_up(off + pb, 256);
+    const size_t o_tok = off;  off = align_up(off + 4 * S * K, 256);
+    const size_t o_cont = off; off = align_up(off + S, 256);
+    const size_t o_acc = off;  off = align_up(off + 4 * S, 256);
+    const size_t o_next = off; off = align_up(off + 4 * S, 256);
+    if (h->stage_bytes < off) {
+        if (h->d_stage) { cudaFree(h->d_stage); h->d_stage = nullptr; h->stage_bytes = 0; }
+        if (cudaMalloc(&h->d_stage, off) != cudaSuccess) { cudaGetLastError(); return TAPOUT_E_ALLOC; }
+        h->stage_bytes = off;
+    }
+    char* d = h->d_stage;
+    int32_t* d_tok = reinterpret_cast<int32_t*>(d + o_tok);
+    uint8_t* d_cont = reinterpret_cast<uint8_t*>(d + o_cont);
+    int32_t* d_acc = reinterpret_cast<int32_t*>(d + o_acc);
+    int32_t* d_next = reinterpret_cast<int32_t*>(d + o_next);
+    TP_CUDA(h, cudaMemsetAsync(d_tok, 0xff, 4 * S * K, h->stream));        // -1 beyond the drafted length
+    TP_CUDA(h, cudaMemcpyAsync(d + o_q, draft_logits, qb, cudaMemcpyHostToDevice, h->stream));
+    TP_CUDA(h, cudaMemcpyAsync(d + o_p, target_logits, pb, cudaMemcpyHostToDevice, h->stream));
+    for (int i = 0; i < p.K; ++i) {
+        int rc = draft_step_impl(h, d + o_q + (size_t)i * V * esz, (int64_t)(K * V), d_tok + i, (int64_t)K, d_cont);
+        if (rc != TAPOUT_OK) return rc;
+    }
+    int rc = verify_impl(h, d + o_q, (int64_t)(K * V), (int64_t)V, d + o_p, (int64_t)((K + 1) * V), (int64_t)V, d_tok,
+                         d_acc, d_next);
+    if (rc != TAPOUT_OK) return rc;
+    rc = update_impl(h);
+    if (rc != TAPOUT_OK) return rc;
+    TP_CUDA(h, cudaMemcpyAsync(out_draft_tokens, d_tok, 4 * S * K, cudaMemcpyDeviceToHost, h->stream));
+    TP_CUDA(h, cudaMemcpyAsync(out_accept_len, d_acc, 4 * S, cudaMemcpyDeviceToHost, h->stream));
+    TP_CUDA(h, cudaMemcpyAsync(out_next_token, d_next, 4 * S, cudaMemcpyDeviceToHost, h->stream));
+    TP_CUDA(h, cudaStreamSynchronize(h->stream));
+    return TAPOUT_OK;
+}
+
+int tapout_row_stats(tapout_t* h, const void* logits, int n_rows, int64_t row_stride, double inv_temp, float* out_features) {
+    if (!h || !logits || !out_features || n_rows < 1 || n_rows > h->p.S) return TAPOUT_E_INVALID_ARG;
+    if (!(inv_temp > 0.0)) return TAPOUT_E_INVALID_ARG;
+    if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
+    if (!aligned16(logits) || !stride_ok(h, row_stride) || row_stride < h->p.V) return TAPOUT_E_ALIGNMENT;
+    const float c = c_of((float)inv_temp);
+    const long long items = (long long)n_rows * h->p.nseg;
+    const int grid = (int)(items < h->grid_rows ? items : h->grid_rows);
+    if (h->p.dtype == DT_BF16)
+        k_draft_rows<DT_BF16><<<grid, kThreads, 0, h->stream>>>(h->p, h->sc, logits, row_stride, 0, n_rows, c);
+    else
+        k_draft_rows<DT_FP32><<<grid, kThreads, 0, h->stream>>>(h->p, h->sc, logits, row_stride, 0, n_rows, c);
+    TP_LAUNCHED(h);
+    k_rows_features<<<(n_rows + 3) / 4, 128, 0, h->stream>>>(h->p, h->sc, n_rows, c, (float)inv_temp, out_features);
+    TP_LAUNCHED(h);
+    return TAPOUT_OK;
+}
+
+int tapout_state_bytes(const tapout_t* h, size_t* bytes) {
+    if (!h || !bytes) return TAPOUT_E_INVALID_ARG;
+    *bytes = h->state_bytes;
+    return TAPOUT_OK;
+}
+
+int tapout_state_field(const tapout_t* h, const char* name, size_t* offset, size_t* bytes) {
+    if (!h || !name) return TAPOUT_E_INVALID_ARG;
+    for (const Field& f : h->fields)
+        if (std::strcmp(f.name, name) == 0) {
+            if (offset) *offset = f.offset;
+            if (bytes) *bytes = f.bytes;
+            return TAPOUT_OK;
+        }
+    return TAPOUT_E_INVALID_ARG;
+}
+
+int tapout_get_state(tapout_t* h, void* host_dst) {
+    if (!h || !host_dst) return TAPOUT_E_INVALID_ARG;
+    TP_CUDA(h, cudaMemcpyAsync(host_dst, h->d_state, h->state_bytes, cudaMemcpyDeviceToHost, h->stream));
+    TP_CUDA(h, cudaStreamSynchronize(h->stream));
+    return TAPOUT_OK;
+}
+
+int tapout_set_state(tapout_t* h, const void* host_src) {
+    if (!h || !host_src) return TAPOUT_E_INVALID_ARG;
+    TP_CUDA(h, cudaMemcpyAsync(h->d_state, host_src, h->state_bytes, cudaMemcpyHostToDevice, h->stream));
+    if (!h->verified && h->pos < h->p.K) {
+        k_rebuild_active<<<1, 1024, 0, h->stream>>>(h->p, h->st, h->sc, h->pos & 1);
+        TP_LAUNCHED(h);
+    }
+    TP_CUDA(h, cudaStreamSynchronize(h->stream));
+    return TAPOUT_OK;
+}
+
+int tapout_get_round(const tapout_t* h, uint32_t* round, int32_t* pos) {
+    if (!h) return TAPOUT_E_INVALID_ARG;
+    if (round) *round = h->round;
+    if (pos) *pos = h->pos;
+    return TAPOUT_OK;
+}
+
+int tapout_set_round(tapout_t* h, uint32_t round) {
+    if (!h) return TAPOUT_E_INVALID_ARG;
+    if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
+    h->round = round;
+    return TAPOUT_OK;
+}
+
+int tapout_get_status(tapout_t* h, uint64_t* bits, uint64_t* rows_draft, uint64_t* rows_target, uint64_t* rows_residual) {
+    if (!h) return TAPOUT_E_INVALID_ARG;
+    unsigned long long v[4];
+    TP_CUDA(h, cudaMemcpyAsync(v, h->sc.status, sizeof v, cudaMemcpyDeviceToHost, h->stream));
+    TP_CUDA(h, cudaStreamSynchronize(h->stream));
+    if (bits) *bits = v[0];
+    if (rows_draft) *rows_draft = v[1];
+    if (rows_target) *rows_target = v[2];
+    if (rows_residual) *rows_residual = v[3];
+    return TAPOUT_OK;
+}
+
+int tapout_get_profile(tapout_t* h, int kernel, double* ms, uint64_t* launches, int reset) {
+    if (!h || kernel < 0 || kernel > 1) return TAPOUT_E_INVALID_ARG;
+    if (h->ev[kernel].size() % 2 != 0) return TAPOUT_E_BAD_STATE;
+    int rc = drain_profile(h, kernel);
+    if (rc != TAPOUT_OK) return rc;
+    if (ms) *ms = h->prof_ms[kernel];
+    if (launches) *launches = h->prof_n[kernel];
+    if (reset) { h->prof_ms[kernel] = 0.0; h->prof_n[kernel] = 0; }
+    return TAPOUT_OK;
+}
+
+int tapout_get_launch_count(const tapout_t* h, uint64_t* launches) {
+    if (!h || !launches) return TAPOUT_E_INVALID_ARG;
+    *launches = h->launches;
+    return TAPOUT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,479 @@
+// Device-side building blocks of libtapout (sm_100a): Philox, 128-bit row loads,
+// one-pass softmax sums per 2 KB warp chunk, CDF search over chunk partials, bandit math.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+namespace tpo {
+
+constexpr int kThreads = 256;            // CTA size of the streaming kernels
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxArms = 16;
+constexpr int kFeat = 6;                 // m, lse, p1, p2, H, argmax
+constexpr int kVecPerLane = 4;           // 16-byte loads per lane and chunk -> 2 KB per warp chunk
+constexpr int kMaxSeg = 32;              // CTAs sharing one row (one lane per segment in the finish)
+constexpr double kLog2e = 1.4426950408889634074;
+constexpr double kLn2 = 0.6931471805599453094;
+
+enum { DT_FP32 = 0, DT_BF16 = 1 };
+enum { RNG_DRAFT = 0, RNG_ACCEPT = 1, RNG_RESAMPLE = 2, RNG_BANDIT = 3 };
+
+template <int DT> struct Elem;
+template <> struct Elem<DT_FP32> { static constexpr int PV = 4; static constexpr int BYTES = 4; };
+template <> struct Elem<DT_BF16> { static constexpr int PV = 8; static constexpr int BYTES = 2; };
+template <int DT> __host__ __device__ constexpr int chunk_elems() { return 32 * kVecPerLane * Elem<DT>::PV; }
+
+// Everything a kernel needs to know about the problem; passed by value.
+struct Params {
+    int S, V, K, A, P, policy, level, dtype;
+    int rule_of_arm[kMaxArms];
+    uint32_t seed_lo, seed_hi, seq_offset;
+    float inv_Tq, inv_Tp;
+    double h_maxconf, h_svip, h_diff, h_margin;
+    double ada_gamma, ada_alpha, ada_beta1, ada_beta2, ada_eps, ada_lambda0, ada_acc0;
+    double reward_alpha, ucb_c2, ts_mu0, ts_var0, ts_noise_var;
+    uint32_t ts_a0, ts_b0;
+    int reward_kind, token_update_all;
+    int nseg, NC;                        // CTAs per draft row, chunks per row
+};
+
+// Pointers into the state blob (SoA; see tapout_state_field).
+struct State {
+    uint32_t* cnt; double* rsum; double* rsum2; double* lambda; double* acc_rate;
+    int32_t* arm; int32_t* n_drafted; int32_t* active; double* sqrtH_prev; double* lse_q;
+    float* feat; int32_t* accept_len; double* reward;
+};
+
+// Partial result of one CTA over its share of a row.
+struct SegRec { float ref, S, T, m2; int argmax; int pad0, pad1, pad2; };
+
+struct Scratch {
+    SegRec* seg;                 // [S][nseg]
+    float2* cdf;                 // [S][NC]: (reference logit, sum of 2^(z*c + k)) per chunk
+    int32_t* list;               // [2][S] sequences still drafting, ping-pong by position parity
+    int32_t* count;              // [0],[1] lengths of the two lists; [2] verify queue head
+    int32_t* order;              // [S] verify order, longest drafts first
+    unsigned long long* status;  // [0] sticky bits, [1] draft rows, [2] target rows, [3] residual rows
+};
+
+// ------------------------------------------------------------------ small helpers
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
+
+// Warp maximum through the integer reduction unit: floats map monotonically to ints.
+__device__ __forceinline__ float warp_max_f(float v) {
+    int i = __float_as_int(v);
+    i ^= (i >> 31) & 0x7fffffff;
+    i = __reduce_max_sync(0xffffffffu, i);
+    i ^= (i >> 31) & 0x7fffffff;
+    return __int_as_float(i);
+}
+
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ double warp_incl_scan_d(double v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        double t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+
+// ------------------------------------------------------------------ Philox4x32-10
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+        c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+        k.x += 0x9E3779B9u;
+        k.y += 0xBB67AE85u;
+    }
+    return c;
+}
+
+__device__ __forceinline__ uint4 rng_words(const Params& p, uint32_t seq, uint32_t round, uint32_t pos,
+                                           uint32_t purpose, uint32_t arm, uint32_t draw) {
+    return philox4x32_10(make_uint4(seq, round, pos, (purpose & 15u) | ((arm & 15u) << 4) | (draw << 8)),
+                         make_uint2(p.seed_lo, p.seed_hi));
+}
+
+__device__ __forceinline__ double u24_to_double(uint32_t word) { return (double)(word >> 8) * (1.0 / 16777216.0); }
+
+// ------------------------------------------------------------------ row access
+template <int DT> __device__ __forceinline__ float load_elem(const void* row, int idx);
+template <> __device__ __forceinline__ float load_elem<DT_FP32>(const void* row, int idx) {
+    return __ldg(reinterpret_cast<const float*>(row) + idx);
+}
+template <> __device__ __forceinline__ float load_elem<DT_BF16>(const void* row, int idx) {
+    const uint32_t b = __ldg(reinterpret_cast<const unsigned short*>(row) + idx);
+    return __uint_as_float(b << 16);
+}
+
+// One warp chunk = 4 x 16 bytes per lane, lane-interleaved so every load instruction covers 512
+// contiguous bytes.  Elements at or beyond V read as -inf.  The row base is 16-byte aligned.
+template <int DT>
+__device__ __forceinline__ void load_chunk(const void* row, int V, int ch, int lane, uint4 (&v)[kVecPerLane]) {
+    constexpr int PV = Elem<DT>::PV;
+    constexpr int CH = chunk_elems<DT>();
+    const int base = ch * CH;
+    const uint4* rp = reinterpret_cast<const uint4*>(row);
+    if (base + CH <= V) {
+#pragma unroll
+        for (int j = 0; j < kVecPerLane; ++j) v[j] = __ldg(rp + base / PV + j * 32 + lane);
+    } else {
+        const uint32_t fill = (DT == DT_BF16) ? 0xff80ff80u : 0xff800000u;
+#pragma unroll
+        for (int j = 0; j < kVecPerLane; ++j) {
+            const int e0 = base + (j * 32 + lane) * PV;
+            if (e0 + PV <= V) {
+                v[j] = __ldg(rp + e0 / PV);
+            } else {
+                uint32_t w[4] = {fill, fill, fill, fill};
+                if (DT == DT_BF16) {
+                    const unsigned short* hp = reinterpret_cast<const unsigned short*>(row);
+                    for (int k = 0; k < PV; ++k)
+                        if (e0 + k < V) {
+                            const uint32_t b = __ldg(hp + e0 + k);
+                            const int sh = (k & 1) * 16;
+                            w[k >> 1] = (w[k >> 1] & ~(0xffffu << sh)) | (b << sh);
+                        }
+                } else {
+                    const uint32_t* fp = reinterpret_cast<const uint32_t*>(row);
+                    for (int k = 0; k < PV; ++k)
+                        if (e0 + k < V) w[k] = __ldg(fp + e0 + k);
+                }
+                v[j] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t x) {
+    __nv_bfloat162 r;
+    *reinterpret_cast<uint32_t*>(&r) = x;
+    return r;
+}
+__device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 x) { return *reinterpret_cast<uint32_t*>(&x); }
+
+// Largest element of the lane's 4 vectors (NaN entries are skipped; they surface in the sums).
+template <int DT> __device__ __forceinline__ float lane_max(const uint4 (&v)[kVecPerLane]);
+template <> __device__ __forceinline__ float lane_max<DT_BF16>(const uint4 (&v)[kVecPerLane]) {
+    __nv_bfloat162 m = as_bf162(v[0].x);
+    m = __hmax2(m, as_bf162(v[0].y)); m = __hmax2(m, as_bf162(v[0].z)); m = __hmax2(m, as_bf162(v[0].w));
+#pragma unroll
+    for (int j = 1; j < kVecPerLane; ++j) {
+        m = __hmax2(m, as_bf162(v[j].x)); m = __hmax2(m, as_bf162(v[j].y));
+        m = __hmax2(m, as_bf162(v[j].z)); m = __hmax2(m, as_bf162(v[j].w));
+    }
+    const uint32_t b = as_u32(m);
+    return fmaxf(__uint_as_float(b << 16), __uint_as_float(b & 0xffff0000u));
+}
+template <> __device__ __forceinline__ float lane_max<DT_FP32>(const uint4 (&v)[kVecPerLane]) {
+    float m = neg_inf();
+#pragma unroll
+    for (int j = 0; j < kVecPerLane; ++j) {
+        m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(v[j].x), __uint_as_float(v[j].y)),
+                           fmaxf(__uint_as_float(v[j].z), __uint_as_float(v[j].w))));
+    }
+    return m;
+}
+
+// sum_e 2^(z_e*c + k) over the lane's elements, and with WANT_T also sum_e w_e*t_e (t_e = z_e*c + k),
+// the numerator of the entropy.  -inf logits are clamped to a huge negative finite value first so that
+// their 0 * (-inf) does not poison the entropy sum; NaN stays NaN.
+template <int DT, bool WANT_T>
+__device__ __forceinline__ void lane_sums(const uint4 (&v)[kVecPerLane], float c, float k, float& s_out, float& t_out) {
+    float s0 = 0.f, s1 = 0.f, t0 = 0.f, t1 = 0.f;
+    if (DT == DT_BF16) {
+        const __nv_bfloat162 floor2 = as_bf162(0xf149f149u);     // about -1e30 in both halves
+#pragma unroll
+        for (int j = 0; j < kVecPerLane; ++j) {
+            const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t x = w[q];
+                if (WANT_T) x = as_u32(__hmax2_nan(as_bf162(x), floor2));
+                const float a = fmaf(__uint_as_float(x << 16), c, k);
+                const float b = fmaf(__uint_as_float(x & 0xffff0000u), c, k);
+                const float wa = ex2_approx(a), wb = ex2_approx(b);
+                s0 += wa; s1 += wb;
+                if (WANT_T) { t0 = fmaf(wa, a, t0); t1 = fmaf(wb, b, t1); }
+            }
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < kVecPerLane; ++j) {
+            const float z[4] = {__uint_as_float(v[j].x), __uint_as_float(v[j].y), __uint_as_float(v[j].z),
+                                __uint_as_float(v[j].w)};
+#pragma unroll
+            for (int q = 0; q < 4; q += 2) {
+                float a = fmaf(z[q], c, k), b = fmaf(z[q + 1], c, k);
+                if (WANT_T) { a = (a < -1e30f) ? -1e30f : a; b = (b < -1e30f) ? -1e30f : b; }
+                const float wa = ex2_approx(a), wb = ex2_approx(b);
+                s0 += wa; s1 += wb;
+                if (WANT_T) { t0 = fmaf(wa, a, t0); t1 = fmaf(wb, b, t1); }
+            }
+        }
+    }
+    s_out = s0 + s1;
+    t_out = t0 + t1;
+}
+
+// Per-warp running state of the one-pass softmax: reference logit (warp-uniform running maximum),
+// lane-private sums relative to it, and the two largest chunk maxima seen (with multiplicity).
+struct WarpAcc {
+    float ref, k, S, T, c1, c2;
+    int best;
+    __device__ __forceinline__ void init() {
+        ref = neg_inf(); k = 0.f; S = 0.f; T = 0.f; c1 = neg_inf(); c2 = neg_inf(); best = -1;
+    }
+};
+
+// Folds one chunk into acc.  Returns the warp-wide sum of 2^(z*c + acc.k) over the chunk if
+// WANT_PART (all lanes get it), else 0.
+template <int DT, bool WANT_T, bool WANT_PART>
+__device__ __forceinline__ float fold_chunk(WarpAcc& acc, const uint4 (&v)[kVecPerLane], int ch, float c) {
+    const float M = warp_max_f(lane_max<DT>(v));
+    if (M > acc.c1) { acc.c2 = acc.c1; acc.c1 = M; acc.best = ch; }
+    else if (M > acc.c2) { acc.c2 = M; }
+    if (M > acc.ref || M != M) {
+        const float kn = __fmul_rn(-M, c);
+        if (acc.ref > neg_inf()) {
+            const float dd = kn - acc.k;                  // <= 0, exact
+            const float f = ex2_approx(dd);
+            if (WANT_T) acc.T = f * fmaf(dd, acc.S, acc.T);
+            acc.S *= f;
+        }
+        acc.ref = M;
+        acc.k = kn;
+    }
+    if (acc.ref == neg_inf()) return 0.f;                  // nothing finite yet (a NaN reference falls through on purpose)
+    float sc, tc;
+    lane_sums<DT, WANT_T>(v, c, acc.k, sc, tc);
+    acc.S += sc;
+    if (WANT_T) acc.T += tc;
+    return WANT_PART ? warp_sum_f(sc) : 0.f;
+}
+
+// ------------------------------------------------------------------ CDF search over chunk partials
+// contribution of chunk ch to the row total, relative to the row maximum m (mc = m*c in double):
+//   scaled  : part.y * 2^-(k_ch + mc), k_ch = fl(-part.x * c) exactly as the streaming pass used it
+//   absolute: part.y
+__device__ __forceinline__ double chunk_contrib(const float2* part, int ch, float c, double mc, bool scaled) {
+    const float2 p = part[ch];
+    if (!scaled) return (double)p.y;
+    if (!(p.y > 0.f)) return (p.y != p.y) ? (double)p.y : 0.0;
+    const double k = (double)__fmul_rn(-p.x, c);
+    return (double)p.y * exp2(-(k + mc));
+}
+
+struct CdfTotals { double lane_sum, incl, W; };
+
+// Each lane owns a contiguous block of chunks, so the scan is in token order.
+__device__ __forceinline__ CdfTotals cdf_totals(const float2* part, int NC, float c, double mc, bool scaled, int lane) {
+    const int per = (NC + 31) / 32;
+    const int b = lane * per, e = min(NC, b + per);
+    double ls = 0.0;
+    for (int ch = b; ch < e; ++ch) ls += chunk_contrib(part, ch, c, mc, scaled);
+    CdfTotals t;
+    t.lane_sum = ls;
+    t.incl = warp_incl_scan_d(ls, lane);
+    t.W = __shfl_sync(0xffffffffu, t.incl, 31);
+    return t;
+}
+
+// The chunk in which the running sum first exceeds tgt, and tgt minus the sum before that chunk.
+__device__ __forceinline__ int cdf_locate(const float2* part, int NC, float c, double mc, bool scaled, int lane,
+                                          const CdfTotals& t, double tgt, double& rem) {
+    const int per = (NC + 31) / 32;
+    const unsigned over = __ballot_sync(0xffffffffu, t.incl > tgt);
+    const unsigned pos = __ballot_sync(0xffffffffu, t.lane_sum > 0.0);
+    int L;
+    if (over) L = __ffs(over) - 1;
+    else if (pos) L = 31 - __clz(pos);
+    else { rem = 0.0; return -1; }
+    const double excl = __shfl_sync(0xffffffffu, t.incl - t.lane_sum, L);
+    const int b = L * per, e = min(NC, b + per);
+    double run = excl;
+    int pick = -1, last_pos = -1;
+    double before = excl, before_last = excl;
+    for (int ch = b; ch < e; ++ch) {
+        const double x = chunk_contrib(part, ch, c, mc, scaled);
+        if (x > 0.0) { last_pos = ch; before_last = run; }
+        if (run + x > tgt) { pick = ch; before = run; break; }
+        run += x;
+    }
+    if (pick < 0) { pick = last_pos; before = before_last; }
+    rem = tgt - before;
+    return pick;
+}
+
+// Token inside one chunk: weights recomputed in double, 32 tokens per step, token order.
+// WeightFn(idx) -> double weight of token idx (>= 0).  rem is in the same units.
+template <int CH, typename WeightFn>
+__device__ __forceinline__ int pick_in_chunk(int chunk, int V, double rem, int lane, WeightFn wf) {
+    const int base = chunk * CH;
+    double run = 0.0;
+    int last_pos = -1;
+    for (int i = 0; i < CH / 32; ++i) {
+        const int idx = base + i * 32 + lane;
+        if (base + i * 32 >= V) break;
+        const double w = (idx < V) ? wf(idx) : 0.0;
+        const unsigned posm = __ballot_sync(0xffffffffu, w > 0.0);
+        if (posm) last_pos = base + i * 32 + 31 - __clz(posm);
+        const double incl = warp_incl_scan_d(w, lane);
+        const unsigned over = __ballot_sync(0xffffffffu, run + incl > rem);
+        if (over) return base + i * 32 + __ffs(over) - 1;
+        run += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    return last_pos;
+}
+
+// ------------------------------------------------------------------ bandits (double, one thread)
+__device__ __forceinline__ int argmax_first(const double* val, int A) {
+    int best = 0;
+    for (int a = 1; a < A; ++a) if (val[a] > val[best]) best = a;
+    return best;
+}
+
+// UCB1 (Section 3.3): mu_a + sqrt(c2 ln t / N_a), t = 1 + sum N; unplayed arms first.
+__device__ inline int ucb1_select(const uint32_t* N, const double* R, int A, double c2) {
+    for (int a = 0; a < A; ++a) if (N[a] == 0) return a;
+    unsigned long long t = 1;
+    for (int a = 0; a < A; ++a) t += N[a];
+    const double lt = log((double)t);
+    double val[kMaxArms];
+    for (int a = 0; a < A; ++a) val[a] = R[a] / (double)N[a] + sqrt(c2 * lt / (double)N[a]);
+    return argmax_first(val, A);
+}
+
+// UCB-Tuned (Section 3.3): mu_a + sqrt((ln t / N_a) min(1/4, V_a)), V_a = var_a + sqrt(2 ln t / N_a).
+__device__ inline int ucb_tuned_select(const uint32_t* N, const double* R, const double* R2, int A) {
+    for (int a = 0; a < A; ++a) if (N[a] == 0) return a;
+    unsigned long long t = 1;
+    for (int a = 0; a < A; ++a) t += N[a];
+    const double lt = log((double)t);
+    double val[kMaxArms];
+    for (int a = 0; a < A; ++a) {
+        const double n = (double)N[a];
+        const double mu = R[a] / n;
+        const double var = R2[a] / n - mu * mu;
+        const double Va = var + sqrt(2.0 * lt / n);
+        const double cap = Va < 0.25 ? Va : 0.25;
+        val[a] = mu + sqrt((lt / n) * cap);
+    }
+    return argmax_first(val, A);
+}
+
+// Gaussian Thompson Sampling (sequence level): conjugate normal posterior, Box-Muller draw.
+__device__ inline int ts_gauss_select(const Params& p, const uint32_t* N, const double* R, uint32_t seq,
+                                      uint32_t round, uint32_t pos) {
+    double val[kMaxArms];
+    for (int a = 0; a < p.A; ++a) {
+        const double var_n = 1.0 / (1.0 / p.ts_var0 + (double)N[a] / p.ts_noise_var);
+        const double mu_n = var_n * (p.ts_mu0 / p.ts_var0 + R[a] / p.ts_noise_var);
+        const uint4 w = rng_words(p, seq, round, pos, RNG_BANDIT, (uint32_t)a, 0);
+        const double u1 = u24_to_double(w.x), u2 = u24_to_double(w.y);
+        const double z = sqrt(-2.0 * log(1.0 - u1)) * cos(6.283185307179586476925 * u2);
+        val[a] = mu_n + sqrt(var_n) * z;
+    }
+    return argmax_first(val, p.A);
+}
+
+// Beta(alpha, beta), integer parameters, as the alpha-th smallest of n = alpha+beta-1 uniforms
+// (24-bit integers; uniform j = word j%4 of Philox draw j/4).  Whole warp; radix select, 8 bits a pass.
+// hist: 256 words of shared memory private to the warp.
+__device__ inline uint32_t beta_order_stat_warp(const Params& p, uint32_t alpha, uint32_t beta, uint32_t seq,
+                                                uint32_t round, uint32_t pos, uint32_t arm, uint32_t* hist, int lane) {
+    const uint32_t n = alpha + beta - 1;
+    const uint32_t calls = (n + 3) / 4;
+    uint32_t k = alpha - 1;                 // 0-based rank still to find among the candidates
+    uint32_t prefix = 0;
+    for (int pass = 0; pass < 3; ++pass) {
+        const int shift = 16 - 8 * pass;
+        for (int b = lane; b < 256; b += 32) hist[b] = 0;
+        __syncwarp();
+        for (uint32_t d = lane; d < calls; d += 32) {
+            const uint4 w = rng_words(p, seq, round, pos, RNG_BANDIT, arm, d);
+            const uint32_t u[4] = {w.x >> 8, w.y >> 8, w.z >> 8, w.w >> 8};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (d * 4 + j >= n) continue;
+                const bool cand = (pass == 0) || ((u[j] >> (shift + 8)) == prefix);
+                if (cand) atomicAdd(&hist[(u[j] >> shift) & 255u], 1u);
+            }
+        }
+        __syncwarp();
+        // bin holding rank k: 8 bins per lane, then a warp scan
+        uint32_t mine = 0;
+        for (int b = 0; b < 8; ++b) mine += hist[lane * 8 + b];
+        uint32_t incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        const unsigned over = __ballot_sync(0xffffffffu, incl > k);
+        const int L = __ffs(over) - 1;
+        uint32_t run = __shfl_sync(0xffffffffu, incl - mine, L);
+        int bin = L * 8;
+        for (int b = 0; b < 8; ++b) {
+            const uint32_t h = hist[L * 8 + b];
+            if (run + h > k) { bin = L * 8 + b; break; }
+            run += h;
+        }
+        k -= run;
+        prefix = (prefix << 8) | (uint32_t)bin;
+        __syncwarp();
+    }
+    return prefix;
+}
+
+// Beta-Bernoulli Thompson Sampling (token level).  Whole warp; every lane returns the arm.
+__device__ inline int ts_beta_select_warp(const Params& p, const uint32_t* N, const double* R, uint32_t seq,
+                                          uint32_t round, uint32_t pos, uint32_t* hist, int lane) {
+    int best = 0;
+    uint32_t best_v = 0;
+    for (int a = 0; a < p.A; ++a) {
+        const uint32_t succ = (uint32_t)R[a];
+        const uint32_t fail = N[a] - succ;
+        const uint32_t v = beta_order_stat_warp(p, p.ts_a0 + succ, p.ts_b0 + fail, seq, round, pos, (uint32_t)a, hist, lane);
+        if (a == 0 || v > best_v) { best = a; best_v = v; }
+    }
+    return best;
+}
+
+// Stop rules of Table 1 (strict inequalities as printed).  Returns true = stop.
+__device__ inline bool rule_stop(const Params& p, int rule, double p1, double p2, double H, double sqrtH_prev,
+                                 bool has_prev, double lambda) {
+    switch (rule) {
+    case 0: return p1 < p.h_maxconf;
+    case 1: return sqrt(H) > p.h_svip;
+    case 2: return 1.0 - sqrt(p.ada_gamma * H) < lambda;
+    case 3: return has_prev && (sqrt(H) - sqrtH_prev > p.h_diff);
+    case 4: return p1 - p2 < p.h_margin;
+    default: return false;
+    }
+}
+
+}  // namespace tpo

@@ -1,0 +1,244 @@
+"""Lockstep parity harness: runs the CUDA library and the CPU oracle round by round on the
+same seeded logits and the same Philox streams and compares every decision.
+
+Discrete decisions (arm, draft token, continue flag, accepted length, final token) must be equal,
+except where the oracle says the deciding quantity is within 1e-6 of its threshold: such a
+difference is counted as a near-threshold flip and the device is resynchronised to the oracle's
+answer (tokens are caller-owned; library state is patched through tapout_get_state/set_state) so
+that later decisions stay comparable.  Float features must agree to 1e-5 relative; bandit
+statistics, rewards and the AdaEDL state must be equal.
+
+Test infrastructure: the only place where the oracle and the binding meet.
+"""
+from dataclasses import dataclass, field
+
+import numpy as np
+import torch
+
+from oracle import oracle as orc
+from paper_2511_02017_b200 import binding as tp
+from paper_2511_02017_b200 import synth_inputs as si
+
+FEAT_RTOL = 1e-5
+FEAT_FLOOR = 1e-2
+FEAT_NAMES = ["m", "lse", "p1", "p2", "H", "argmax"]
+
+
+@dataclass
+class Report:
+    rounds: int = 0
+    decisions: dict = field(default_factory=lambda: dict(token=0, cont=0, accept=0, next=0, arm=0))
+    flips: dict = field(default_factory=lambda: dict(token=0, cont=0, accept=0, next=0, arm=0))
+    failures: list = field(default_factory=list)
+    max_feat_err: float = 0.0
+    rows_dev: int = 0
+    rows_oracle: int = 0
+    mean_drafted: float = 0.0
+    mean_accepted: float = 0.0
+
+    def ok(self):
+        return not self.failures
+
+    def summary(self):
+        return ("rounds=%d decisions=%s flips=%s max_feat_err=%.2e mean_n=%.2f mean_a=%.2f failures=%d" %
+                (self.rounds, self.decisions, self.flips, self.max_feat_err, self.mean_drafted,
+                 self.mean_accepted, len(self.failures)))
+
+
+def policy_codes(w):
+    pol = {"ucb1": (tp.POLICY_UCB1, orc.UCB1), "ts": (tp.POLICY_TS, orc.TS), "ucb_tuned": (tp.POLICY_UCB_TUNED, orc.UCB_TUNED)}[w.policy]
+    lev = {"seq": (tp.LEVEL_SEQ, orc.SEQ), "token": (tp.LEVEL_TOKEN, orc.TOKEN)}[w.level]
+    return pol, lev
+
+
+def make_device(w, **params):
+    (pd, _), (ld, _) = policy_codes(w)
+    dev = tp.Tapout(w.n_seq, w.vocab, w.k_max, w.n_arms, pd, ld,
+                    seed=w.seed, dtype=tp.DTYPE_BF16 if w.dtype == "bf16" else tp.DTYPE_FP32,
+                    inv_temp_draft=1.0 / w.temp_draft, inv_temp_target=1.0 / w.temp_target,
+                    step_row_stride=w.k_max * w.vocab, **params)
+    return dev
+
+
+def make_oracle(w, seq_ids, **params):
+    (_, po), (_, lo) = policy_codes(w)
+    return orc.Oracle(len(seq_ids), w.vocab, w.k_max, w.n_arms, po, lo,
+                      seed=w.seed, dtype=orc.BF16 if w.dtype == "bf16" else orc.FP32,
+                      inv_temp_draft=np.float32(1.0 / w.temp_draft), inv_temp_target=np.float32(1.0 / w.temp_target),
+                      seq_ids=np.asarray(seq_ids, dtype=np.uint32), **params)
+
+
+def _logit_value(bits_row, idx):
+    v = bits_row[idx]
+    if bits_row.dtype == np.uint16:
+        return float(np.array([int(v) << 16], dtype=np.uint32).view(np.float32)[0])
+    return float(v)
+
+
+def _softmax64(bits_row, inv_T):
+    if bits_row.dtype == np.uint16:
+        z = (bits_row.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    else:
+        z = bits_row.astype(np.float64)
+    z = z * float(np.float32(inv_T))
+    z -= z.max()
+    e = np.exp(z)
+    return e / e.sum()
+
+
+def run_lockstep(w, rounds, sample=None, device="cuda", logits_fn=None, dev_params=None, orc_params=None,
+                 first_round=0, dev=None, ora=None, report=None, check_state_every=1):
+    """Runs `rounds` rounds of workload `w`.  `sample`: local sequence indices the oracle follows
+    (default all).  `logits_fn(w, rnd, device) -> (draft, target)` overrides the synthetic generator.
+    Returns (report, dev, ora) so that a caller can continue."""
+    S, K, V = w.n_seq, w.k_max, w.vocab
+    sample = np.arange(S) if sample is None else np.asarray(sorted(sample))
+    sample_t = torch.as_tensor(sample, device=device, dtype=torch.long)
+    own = dev is None
+    if dev is None:
+        dev = make_device(w, **(dev_params or {}))
+        ora = make_oracle(w, sample, **(orc_params or {}))
+    rep = report or Report()
+    gen = logits_fn or si.round_logits
+    tok_step = torch.empty(S, dtype=torch.int32, device=device)
+    cont_step = torch.empty(S, dtype=torch.uint8, device=device)
+    acc_d = torch.empty(S, dtype=torch.int32, device=device)
+    nxt_d = torch.empty(S, dtype=torch.int32, device=device)
+    inv_Tq, inv_Tp = 1.0 / w.temp_draft, 1.0 / w.temp_target
+    sum_n = sum_a = 0
+
+    def fail(msg):
+        rep.failures.append(msg)
+
+    for rnd in range(first_round, first_round + rounds):
+        draft, target = gen(w, rnd, device)
+        Dn = si.to_numpy_bits(draft[sample_t])
+        Tn = si.to_numpy_bits(target[sample_t])
+        toks = torch.full((S, K), -1, dtype=torch.int32, device=device)
+        toks_o = np.full((len(sample), K), -1, np.int32)
+
+        # ------------------------------------------------------------ draft loop
+        for i in range(K):
+            dev.draft_step(draft[:, i, :], tok_step, cont_step)
+            r = ora.draft_step(Dn[:, i, :])
+            toks[:, i] = tok_step
+            toks_o[:, i] = r["token"]
+            dt = tok_step[sample_t].cpu().numpy()
+            dc = cont_step[sample_t].cpu().numpy()
+            patch_state = []
+            for j in range(len(sample)):
+                ot, oc = int(r["token"][j]), int(r["cont"][j])
+                if ot < 0 and int(dt[j]) < 0:
+                    if int(dc[j]) != 0 or oc != 0:
+                        fail("r%d i%d s%d: stopped sequence has continue=1" % (rnd, i, sample[j]))
+                    continue
+                rep.decisions["token"] += 1
+                rep.decisions["cont"] += 1
+                if int(dt[j]) != ot:
+                    lo, hi = int(r["tok_lo"][j]), int(r["tok_hi"][j])
+                    if ot >= 0 and lo <= int(dt[j]) <= hi and np.isfinite(_logit_value(Dn[j, i], int(dt[j]))):
+                        rep.flips["token"] += 1
+                        toks[int(sample[j]), i] = ot
+                    else:
+                        fail("r%d i%d s%d: token dev=%d oracle=%d band=[%d,%d]" % (rnd, i, sample[j], dt[j], ot, lo, hi))
+                if int(dc[j]) != oc:
+                    if r["near_rule"][j]:
+                        rep.flips["cont"] += 1
+                        patch_state.append((int(sample[j]), oc))
+                    else:
+                        fail("r%d i%d s%d: continue dev=%d oracle=%d" % (rnd, i, sample[j], dc[j], oc))
+            if patch_state:
+                st = dev.get_state()
+                for s_loc, oc in patch_state:
+                    st["active"][s_loc] = oc
+                    st["n_drafted"][s_loc] = i + 1
+                dev.set_state(st)
+
+        # ------------------------------------------------------------ state before verify
+        st = dev.get_state()
+        n_o = ora.view("n_drafted")
+        arms_o = ora.view("arm")
+        feat_o = ora.view("feat")
+        dirty = False
+        for j, s_loc in enumerate(sample):
+            n = int(n_o[j])
+            if int(st["n_drafted"][s_loc]) != n:
+                fail("r%d s%d: n_drafted dev=%d oracle=%d" % (rnd, s_loc, st["n_drafted"][s_loc], n))
+                continue
+            n_arm = n if w.level == "token" else min(n, 1)
+            for i in range(n_arm):
+                rep.decisions["arm"] += 1
+                if int(st["arm"][s_loc, i]) != int(arms_o[j, i]):
+                    fail("r%d s%d i%d: arm dev=%d oracle=%d" % (rnd, s_loc, i, st["arm"][s_loc, i], arms_o[j, i]))
+            for i in range(n):
+                fo, fd = feat_o[j, i], st["feat"][s_loc, i].astype(np.float64)
+                err = np.abs(fd[:5] - fo[:5]) / np.maximum(np.abs(fo[:5]), FEAT_FLOOR)
+                rep.max_feat_err = max(rep.max_feat_err, float(err.max()))
+                if err.max() > FEAT_RTOL:
+                    fail("r%d s%d i%d: features dev=%s oracle=%s" % (rnd, s_loc, i, fd, fo))
+                if int(fd[5]) != int(fo[5]):
+                    fail("r%d s%d i%d: argmax dev=%d oracle=%d" % (rnd, s_loc, i, fd[5], fo[5]))
+            sum_n += n
+
+        # ------------------------------------------------------------ verify
+        dev.verify(draft, target, toks, acc_d, nxt_d)
+        v = ora.verify(Dn, Tn, toks_o)
+        da = acc_d[sample_t].cpu().numpy()
+        dn = nxt_d[sample_t].cpu().numpy()
+        patch_acc = []
+        for j, s_loc in enumerate(sample):
+            oa, on = int(v["accept_len"][j]), int(v["next_token"][j])
+            rep.decisions["accept"] += 1
+            sum_a += oa
+            if int(da[j]) != oa:
+                if v["near_accept"][j]:
+                    rep.flips["accept"] += 1
+                    patch_acc.append((int(s_loc), oa))
+                else:
+                    fail("r%d s%d: accept_len dev=%d oracle=%d" % (rnd, s_loc, da[j], oa))
+                continue
+            rep.decisions["next"] += 1
+            if int(dn[j]) != on:
+                lo, hi = int(v["next_lo"][j]), int(v["next_hi"][j])
+                okband = on >= 0 and lo <= int(dn[j]) <= hi
+                if okband:
+                    p = _softmax64(Tn[j, oa], inv_Tp)
+                    if oa < int(n_o[j]):
+                        q = _softmax64(Dn[j, oa], inv_Tq)
+                        okband = (p[int(dn[j])] - q[int(dn[j])]) > 0
+                    else:
+                        okband = p[int(dn[j])] > 0
+                if okband:
+                    rep.flips["next"] += 1
+                else:
+                    fail("r%d s%d: next_token dev=%d oracle=%d band=[%d,%d] a=%d" % (rnd, s_loc, dn[j], on, lo, hi, oa))
+        if patch_acc:
+            st = dev.get_state()
+            for s_loc, oa in patch_acc:
+                st["accept_len"][s_loc] = oa
+            dev.set_state(st)
+
+        # ------------------------------------------------------------ update
+        dev.update()
+        ora.update()
+        if (rnd - first_round) % check_state_every == 0 or rnd == first_round + rounds - 1:
+            st = dev.get_state()
+            for name in ("cnt", "rsum", "rsum2", "lambda", "acc_rate", "reward"):
+                a = st[name][sample]
+                b = ora.view(name)
+                if not np.array_equal(a, b):
+                    bad = np.argwhere(np.asarray(a != b))[0]
+                    fail("r%d: state %s differs at %s: dev=%r oracle=%r" % (rnd, name, bad.tolist(), a[tuple(bad)], b[tuple(bad)]))
+        rep.rounds += 1
+        if len(rep.failures) > 20:
+            break
+
+    stt = dev.get_status()
+    rep.rows_dev = stt["rows_draft"] + stt["rows_target"] + stt["rows_residual"]
+    rep.rows_oracle = ora.rows_read
+    nd = max(1, rep.decisions["accept"])
+    rep.mean_drafted = sum_n / nd
+    rep.mean_accepted = sum_a / nd
+    if own and report is None:
+        pass
+    return rep, dev, ora

@@ -1,0 +1,396 @@
+"""GPU parity tests: the CUDA library (through the C ABI binding) against the CPU oracle on the
+same seeded inputs.  Run with `pytest -m gpu` on a B200."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2511_02017_b200 import binding as tp
+from paper_2511_02017_b200 import synth_inputs as si
+from tests.lockstep import FEAT_FLOOR, FEAT_RTOL, run_lockstep
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _assert_clean(rep, max_flip_rate=0.05):
+    assert rep.ok(), "\n".join(rep.failures[:10]) + "\n" + rep.summary()
+    for k, n in rep.decisions.items():
+        if n >= 200:
+            assert rep.flips[k] <= max_flip_rate * n, rep.summary()
+    assert rep.max_feat_err <= FEAT_RTOL
+    print(rep.summary())
+
+
+def peaked_logits(w, rnd, device):
+    """The workload's rows with one token per row lifted by U[6,16]: top-1 probabilities then spread over
+    (0,1) so that every stop rule fires on some rows and drafts of every length occur."""
+    d, t = si.round_logits(w, rnd, device)
+    g = torch.Generator(device="cpu")
+    g.manual_seed(1234 + rnd)
+    S, K, V = w.n_seq, w.k_max, w.vocab
+    idx = torch.randint(0, V, (S, K + 1), generator=g).to(device)
+    lift = (6 + 10 * torch.rand((S, K + 1), generator=g)).to(device)
+    tt = t.float()
+    tt.scatter_add_(2, idx.unsqueeze(-1), lift.unsqueeze(-1))
+    dd = d.float()
+    dd.scatter_add_(2, idx[:, :K].unsqueeze(-1), (lift[:, :K] * 0.9).unsqueeze(-1))
+    return dd.to(d.dtype), tt.to(t.dtype)
+
+
+# ------------------------------------------------------------------ row statistics kernel
+def _rows_case(dtype):
+    rng = np.random.default_rng(0)
+    V = 5001 if dtype == "fp32" else 9003        # several chunks, ragged tail, not a multiple of the vector width
+    rows = []
+    rows.append(np.zeros(V))                                                    # uniform
+    z = np.zeros(V); z[V - 1] = 7.0; rows.append(z)                             # one-hot at the very end
+    z = rng.normal(size=V) * 3; z[17] = z[4021] = z.max() + 1.0; rows.append(z)  # duplicated maximum
+    z = rng.normal(size=V) * 3; z[::3] = -np.inf; rows.append(z)                # -inf entries
+    z = np.full(V, -np.inf); z[123] = 0.5; rows.append(z)                       # a single finite entry
+    z = rng.normal(size=V) * 3; z[100] = np.nan; rows.append(z)                 # NaN -> unusable
+    rows.append(np.full(V, -np.inf))                                            # no finite entry -> unusable
+    z = rng.normal(size=V) * 3; z[5] = np.inf; rows.append(z)                   # +inf -> unusable
+    z = rng.normal(size=V) * 30; rows.append(z)                                 # very peaked
+    z = rng.normal(size=V) * 0.01 + 80.0; rows.append(z)                        # large offset
+    for _ in range(6):
+        rows.append(rng.normal(size=V) * 3 - 1.1 * np.log1p(rng.permutation(V)))
+    return V, np.stack(rows).astype(np.float32)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("inv_T", [1.0, 1.0 / 0.7])
+def test_row_stats_kernel_against_oracle(dtype, inv_T):
+    V, rows = _rows_case(dtype)
+    n = rows.shape[0]
+    Vs = V + (-V) % 8                                   # row stride: multiple of 16 bytes
+    buf = torch.zeros((n, Vs), dtype=torch.float32)
+    buf[:, :V] = torch.from_numpy(rows)
+    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    dev_rows = buf.to(td).to(DEV)
+    host_bits = si.to_numpy_bits(dev_rows)[:, :V]
+    h = tp.Tapout(n, V, 2, 1, tp.POLICY_UCB1, tp.LEVEL_SEQ, dtype=tp.DTYPE_BF16 if dtype == "bf16" else tp.DTYPE_FP32)
+    for segs in (0, 1, 3):
+        h.set_param("row_segments", segs)
+        out = torch.zeros((n, 6), dtype=torch.float32, device=DEV)
+        h.row_stats(dev_rows, n, Vs, inv_T, out)
+        got = out.cpu().numpy().astype(np.float64)
+        for r in range(n):
+            st = orc.row_stats(np.ascontiguousarray(host_bits[r]), inv_T=np.float32(inv_T))
+            if not st.valid:
+                assert np.all(np.isnan(got[r, :5])) and got[r, 5] == -1, (r, got[r])
+                continue
+            want = np.array([st.m, st.lse, st.p1, st.p2, st.H])
+            err = np.abs(got[r, :5] - want) / np.maximum(np.abs(want), FEAT_FLOOR)
+            assert err.max() <= FEAT_RTOL, (segs, r, got[r], want)
+            assert int(got[r, 5]) == st.argmax, (segs, r)
+    h.destroy()
+
+
+def test_small_vocabularies():
+    # vocab smaller than one chunk / one warp's loads; rows still 16-byte multiples
+    for V in (8, 24, 1032):
+        w = si.Workload("small", 5, V, "bf16", 3, 1, 5, "ucb1", "seq", seed=5)
+        rep, dev, _ = run_lockstep(w, 6, device=DEV)
+        _assert_clean(rep)
+        dev.destroy()
+
+
+@pytest.mark.parametrize("V,Vs", [(2, 8), (7, 8), (33, 40), (1003, 1008)])
+def test_strided_rows_unaligned_vocab(V, Vs):
+    # vocab not a multiple of the vector width: rows padded to a 16-byte multiple, strides passed explicitly
+    S, K = 6, 3
+    w = si.Workload("strided", S, V, "bf16", K, 1, 5, "ucb1", "seq", seed=8)
+    dev = tp.Tapout(S, V, K, 5, tp.POLICY_UCB1, tp.LEVEL_SEQ, seed=8, step_row_stride=K * Vs, q_seq_stride=K * Vs,
+                    q_pos_stride=Vs, p_seq_stride=(K + 1) * Vs, p_pos_stride=Vs)
+    ora = orc.Oracle(S, V, K, 5, orc.UCB1, orc.SEQ, seed=8, dtype=orc.BF16)
+    tok = torch.empty(S, dtype=torch.int32, device=DEV)
+    cont = torch.empty(S, dtype=torch.uint8, device=DEV)
+    acc = torch.empty(S, dtype=torch.int32, device=DEV)
+    nxt = torch.empty(S, dtype=torch.int32, device=DEV)
+    for rnd in range(5):
+        d, t = si.round_logits(w, rnd, DEV)
+        dp = torch.full((S, K, Vs), 50.0, dtype=torch.bfloat16, device=DEV)      # padding holds large logits: must be ignored
+        tpad = torch.full((S, K + 1, Vs), 50.0, dtype=torch.bfloat16, device=DEV)
+        dp[:, :, :V] = d
+        tpad[:, :, :V] = t
+        Dn, Tn = si.to_numpy_bits(d), si.to_numpy_bits(t)
+        toks = torch.full((S, K), -1, dtype=torch.int32, device=DEV)
+        toks_o = np.full((S, K), -1, np.int32)
+        for i in range(K):
+            dev.draft_step(dp[:, i, :], tok, cont)
+            r = ora.draft_step(Dn[:, i, :])
+            toks_o[:, i] = r["token"]
+            got = tok.cpu().numpy()
+            band = (r["tok_lo"] <= got) & (got <= r["tok_hi"])
+            assert np.all((got == r["token"]) | band), (got, r["token"])
+            toks[:, i] = torch.from_numpy(r["token"]).to(DEV)
+            assert np.array_equal(cont.cpu().numpy(), r["cont"])
+        dev.verify(dp, tpad, toks, acc, nxt)
+        v = ora.verify(Dn, Tn, toks_o)
+        assert np.array_equal(acc.cpu().numpy(), v["accept_len"])
+        nd = nxt.cpu().numpy()
+        assert np.all((nd == v["next_token"]) | ((v["next_lo"] <= nd) & (nd <= v["next_hi"])))
+        dev.update()
+        ora.update()
+    dev.destroy()
+
+
+# ------------------------------------------------------------------ lockstep on the benchmark workloads
+def test_lockstep_tiny_full():
+    """Config 1 in full: 1 sequence, vocab 32000, fp32, k_max 8, 256 rounds, 3 arms, sequence-level UCB1."""
+    w = si.WORKLOADS["tiny"]
+    rep, dev, _ = run_lockstep(w, w.rounds, device=DEV)
+    _assert_clean(rep)
+    dev.destroy()
+
+
+@pytest.mark.parametrize("name,S,rounds", [("batch64", 12, 8), ("batch256_ts", 10, 8), ("throughput", 16, 6),
+                                           ("shift", 6, 4), ("shift_ts", 6, 4)])
+def test_lockstep_reduced_batch_full_vocab(name, S, rounds):
+    """Configs 2-5 with the full vocabulary, dtype, k_max, bandit and generator, fewer sequences and rounds."""
+    w = si.scaled(si.WORKLOADS[name], n_seq=S)
+    rep, dev, _ = run_lockstep(w, rounds, device=DEV)
+    _assert_clean(rep)
+    assert rep.rows_dev == rep.rows_oracle
+    dev.destroy()
+
+
+@pytest.mark.parametrize("name", ["batch64", "batch256_ts", "throughput"])
+def test_lockstep_peaked_rows_all_rules(name):
+    w = si.scaled(si.WORKLOADS[name], n_seq=12, vocab=20008)
+    rep, dev, _ = run_lockstep(w, 24, device=DEV, logits_fn=peaked_logits)
+    _assert_clean(rep)
+    assert 1.2 < rep.mean_drafted < w.k_max          # drafts of mixed length
+    dev.destroy()
+
+
+@pytest.mark.parametrize("policy,level", [("ucb1", "seq"), ("ts", "seq"), ("ucb1", "token"), ("ts", "token"),
+                                          ("ucb_tuned", "seq"), ("ucb_tuned", "token")])
+def test_all_controllers_many_rounds(policy, level):
+    """The four controllers of the paper (and UCB-Tuned) over enough rounds for the statistics to matter."""
+    w = si.Workload("ctl", 8, 4104, "bf16", 6, 1, 5, policy, level, seed=21, sigma="per_seq:0.2:1.5")
+    rep, dev, _ = run_lockstep(w, 60, device=DEV, logits_fn=peaked_logits)
+    _assert_clean(rep)
+    dev.destroy()
+
+
+def test_reward_simple_and_token_update_switch():
+    w = si.Workload("rs", 8, 4104, "bf16", 6, 1, 5, "ucb1", "seq", seed=22)
+    rep, dev, _ = run_lockstep(w, 20, device=DEV, logits_fn=peaked_logits, dev_params=dict(reward_kind=1),
+                               orc_params=dict(reward_kind=1))
+    _assert_clean(rep)
+    dev.destroy()
+    w = si.Workload("tu", 8, 4104, "bf16", 6, 1, 5, "ucb1", "token", seed=23)
+    rep, dev, _ = run_lockstep(w, 20, device=DEV, logits_fn=peaked_logits, dev_params=dict(token_update_all=0),
+                               orc_params=dict(token_update_all=0))
+    _assert_clean(rep)
+    dev.destroy()
+
+
+def test_static_arm_pool_and_thresholds():
+    w = si.Workload("st", 6, 4104, "fp32", 5, 1, 3, "ucb1", "seq", seed=24)
+    arms = [tp.RULE_STATIC, tp.RULE_SVIP, tp.RULE_MARGIN]
+    rep, dev, _ = run_lockstep(w, 12, device=DEV, logits_fn=peaked_logits,
+                               dev_params=dict(arms=arms, h_svip=0.9, h_margin=0.35),
+                               orc_params=dict(arms=arms, h_svip=0.9, h_margin=0.35))
+    _assert_clean(rep)
+    dev.destroy()
+
+
+@pytest.mark.parametrize("name,rounds,n_sample", [("throughput", 2, 6), ("batch256_ts", 2, 5), ("shift", 1, 4),
+                                                  ("batch64", 2, 6)])
+def test_lockstep_full_size_sampled_sequences(name, rounds, n_sample):
+    """Full-size configs in the launch configuration the benchmark times; the oracle follows a sample of
+    the sequences (sequences are independent, so each is a complete check of its own stream)."""
+    w = si.WORKLOADS[name]
+    rng = np.random.default_rng(3)
+    sample = sorted(rng.choice(w.n_seq, size=n_sample, replace=False).tolist())
+    rep, dev, _ = run_lockstep(w, rounds, sample=sample, device=DEV)
+    _assert_clean(rep, max_flip_rate=0.2)
+    st = dev.get_state()
+    n_all = st["cnt"].sum(axis=(1, 2))
+    if w.level == "seq":
+        assert np.all(n_all == rounds)                # every sequence of the batch was updated every round
+    dev.destroy()
+    torch.cuda.empty_cache()
+
+
+# ------------------------------------------------------------------ invalid rows, API misuse, state
+def test_unusable_rows_follow_the_oracle():
+    S, V, K = 4, 2048, 4
+    w = si.Workload("bad", S, V, "bf16", K, 1, 1, "ucb1", "seq", seed=9)
+
+    def gen(w_, rnd, device):
+        d, t = si.round_logits(w_, rnd, device)
+        d[0, 0, 3] = float("nan")          # nothing can be drafted
+        d[1, 2, :] = float("-inf")         # stops after two tokens
+        t[2, 1, 7] = float("inf")          # target row 1 unusable
+        return d, t
+    arms = [tp.RULE_STATIC]
+    rep, dev, ora = run_lockstep(w, 2, device=DEV, logits_fn=gen, dev_params=dict(arms=arms), orc_params=dict(arms=arms))
+    _assert_clean(rep)
+    bits = dev.get_status()["bits"]
+    assert bits & tp.ST_BAD_DRAFT_ROW and bits & tp.ST_BAD_TARGET_ROW
+    assert ora.status & orc.ST_BAD_DRAFT_ROW and ora.status & orc.ST_BAD_TARGET_ROW
+    dev.destroy()
+
+
+def test_api_misuse_returns_error_codes():
+    L = tp.load()
+    h = C.c_void_p()
+    assert L.tapout_create(C.byref(h), 0, 100, 4, 5, 0, 0) == tp.E_INVALID_ARG
+    assert L.tapout_create(C.byref(h), 4, 100, 4, 17, 0, 0) == tp.E_INVALID_ARG
+    assert L.tapout_create(C.byref(h), 4, 100, 4, 5, 9, 0) == tp.E_INVALID_ARG
+    assert L.tapout_create(None, 4, 100, 4, 5, 0, 0) == tp.E_INVALID_ARG
+    S, V, K = 4, 1024, 3
+    t = tp.Tapout(S, V, K, 5, tp.POLICY_UCB1, tp.LEVEL_SEQ)
+    d = torch.randn((S, K, V), device=DEV).to(torch.bfloat16)
+    p = torch.randn((S, K + 1, V), device=DEV).to(torch.bfloat16)
+    tok = torch.empty(S, dtype=torch.int32, device=DEV)
+    cont = torch.empty(S, dtype=torch.uint8, device=DEV)
+    toks = torch.zeros((S, K), dtype=torch.int32, device=DEV)
+    acc = torch.empty(S, dtype=torch.int32, device=DEV)
+    nxt = torch.empty(S, dtype=torch.int32, device=DEV)
+    assert L.tapout_update(t.h) == tp.E_BAD_STATE
+    assert L.tapout_verify(t.h, d.data_ptr(), p.data_ptr(), toks.data_ptr(), acc.data_ptr(), nxt.data_ptr()) == tp.E_BAD_STATE
+    assert L.tapout_draft_step(t.h, None, tok.data_ptr(), cont.data_ptr()) == tp.E_INVALID_ARG
+    assert L.tapout_draft_step(t.h, d.data_ptr() + 2, tok.data_ptr(), cont.data_ptr()) == tp.E_ALIGNMENT
+    assert L.tapout_set_param_i64(t.h, tp.PARAM["step_row_stride"], V - 8) == tp.E_INVALID_ARG
+    t.set_param("step_row_stride", K * V)
+    for i in range(K):
+        t.draft_step(d[:, i, :], tok, cont)
+    assert L.tapout_draft_step(t.h, d.data_ptr(), tok.data_ptr(), cont.data_ptr()) == tp.E_BAD_STATE
+    assert L.tapout_set_param_f64(t.h, tp.PARAM["h_svip"], 0.5) == tp.E_BAD_STATE          # mid-round
+    assert L.tapout_update(t.h) == tp.E_BAD_STATE
+    t.verify(d, p, toks, acc, nxt)
+    assert L.tapout_verify(t.h, d.data_ptr(), p.data_ptr(), toks.data_ptr(), acc.data_ptr(), nxt.data_ptr()) == tp.E_BAD_STATE
+    t.update()
+    assert t.get_round() == (1, 0)
+    assert L.tapout_set_param_f64(t.h, 999, 0.5) == tp.E_INVALID_ARG
+    assert L.tapout_set_param_f64(t.h, tp.PARAM["inv_temp_draft"], -1.0) == tp.E_INVALID_ARG
+    assert L.tapout_destroy(None) == tp.E_INVALID_ARG
+    torch.cuda.synchronize()
+    t.destroy()
+
+
+def test_out_of_range_draft_token_is_rejected_not_read():
+    S, V, K = 2, 2048, 2
+    t = tp.Tapout(S, V, K, 1, tp.POLICY_UCB1, tp.LEVEL_SEQ, arms=[tp.RULE_STATIC], step_row_stride=K * V)
+    d = torch.randn((S, K, V), device=DEV).to(torch.bfloat16)
+    p = d.new_zeros((S, K + 1, V))
+    p[:, :K] = d
+    tok = torch.empty(S, dtype=torch.int32, device=DEV)
+    cont = torch.empty(S, dtype=torch.uint8, device=DEV)
+    toks = torch.zeros((S, K), dtype=torch.int32, device=DEV)
+    for i in range(K):
+        t.draft_step(d[:, i, :], tok, cont)
+        toks[:, i] = tok
+    toks[1, 0] = V + 5
+    acc = torch.empty(S, dtype=torch.int32, device=DEV)
+    nxt = torch.empty(S, dtype=torch.int32, device=DEV)
+    t.verify(d, p, toks, acc, nxt)
+    assert acc.cpu().tolist() == [K, 0]                 # p == q accepts everything; the bad token is a rejection
+    assert t.get_status()["bits"] & tp.ST_BAD_TOKEN
+    t.update()
+    t.destroy()
+
+
+def test_checkpoint_resume_is_bitwise_equivalent():
+    w = si.Workload("ck", 6, 4104, "bf16", 4, 1, 5, "ucb1", "seq", seed=31)
+
+    def run(dev, rounds, first):
+        outs = []
+        S, K = w.n_seq, w.k_max
+        tok = torch.empty(S, dtype=torch.int32, device=DEV)
+        cont = torch.empty(S, dtype=torch.uint8, device=DEV)
+        acc = torch.empty(S, dtype=torch.int32, device=DEV)
+        nxt = torch.empty(S, dtype=torch.int32, device=DEV)
+        for rnd in range(first, first + rounds):
+            d, t = peaked_logits(w, rnd, DEV)
+            toks = torch.full((S, K), -1, dtype=torch.int32, device=DEV)
+            for i in range(K):
+                dev.draft_step(d[:, i, :], tok, cont)
+                toks[:, i] = tok
+            dev.verify(d, t, toks, acc, nxt)
+            dev.update()
+            outs.append((toks.cpu().numpy().copy(), acc.cpu().numpy().copy(), nxt.cpu().numpy().copy()))
+        return outs
+    from tests.lockstep import make_device
+    a = make_device(w)
+    ref = run(a, 10, 0)
+    b = make_device(w)
+    run(b, 4, 0)
+    blob = b.get_state()
+    b.destroy()
+    c = make_device(w)                                 # a fresh handle resumes from the blob and the round number
+    c.set_round(4)
+    c.set_state(blob)
+    got = run(c, 6, 4)
+    for (t1, a1, n1), (t2, a2, n2) in zip(ref[4:], got):
+        assert np.array_equal(t1, t2) and np.array_equal(a1, a2) and np.array_equal(n1, n2)
+    assert np.array_equal(a.get_state()["_blob"], c.get_state()["_blob"])
+    a.destroy()
+    c.destroy()
+
+
+def test_round_host_matches_device_path():
+    w = si.Workload("host", 5, 4104, "bf16", 4, 1, 5, "ucb1", "seq", seed=41)
+    from tests.lockstep import make_device
+    a, b = make_device(w), make_device(w)
+    S, K = w.n_seq, w.k_max
+    tok = torch.empty(S, dtype=torch.int32, device=DEV)
+    cont = torch.empty(S, dtype=torch.uint8, device=DEV)
+    acc = torch.empty(S, dtype=torch.int32, device=DEV)
+    nxt = torch.empty(S, dtype=torch.int32, device=DEV)
+    for rnd in range(5):
+        d, t = peaked_logits(w, rnd, DEV)
+        toks = torch.full((S, K), -1, dtype=torch.int32, device=DEV)
+        for i in range(K):
+            a.draft_step(d[:, i, :], tok, cont)
+            toks[:, i] = tok
+        a.verify(d, t, toks, acc, nxt)
+        a.update()
+        hd, ht = d.cpu().pin_memory(), t.cpu().pin_memory()
+        o_tok = torch.empty((S, K), dtype=torch.int32).pin_memory()
+        o_acc = torch.empty(S, dtype=torch.int32).pin_memory()
+        o_nxt = torch.empty(S, dtype=torch.int32).pin_memory()
+        b.round_host(hd, ht, o_tok, o_acc, o_nxt)
+        assert torch.equal(o_tok, toks.cpu()) and torch.equal(o_acc, acc.cpu()) and torch.equal(o_nxt, nxt.cpu())
+    sa, sb = a.get_state(), b.get_state()
+    assert np.array_equal(sa["_blob"], sb["_blob"])
+    a.destroy()
+    b.destroy()
+
+
+def test_seq_offset_shards_reproduce_the_full_batch():
+    """Sharding by sequence (one handle per shard, seq_offset = first global id) gives the same streams."""
+    w = si.Workload("shard", 8, 4104, "bf16", 4, 1, 5, "ts", "seq", seed=51)
+    from tests.lockstep import make_device
+    full = make_device(w)
+    halves = [make_device(si.scaled(w, n_seq=4), seq_offset=0), make_device(si.scaled(w, n_seq=4), seq_offset=4)]
+    K = w.k_max
+
+    def round_on(dev, d, t):
+        S = d.shape[0]
+        tok = torch.empty(S, dtype=torch.int32, device=DEV)
+        cont = torch.empty(S, dtype=torch.uint8, device=DEV)
+        acc = torch.empty(S, dtype=torch.int32, device=DEV)
+        nxt = torch.empty(S, dtype=torch.int32, device=DEV)
+        toks = torch.full((S, K), -1, dtype=torch.int32, device=DEV)
+        for i in range(K):
+            dev.draft_step(d[:, i, :], tok, cont)
+            toks[:, i] = tok
+        dev.verify(d, t, toks, acc, nxt)
+        dev.update()
+        return toks.cpu(), acc.cpu(), nxt.cpu()
+    for rnd in range(6):
+        d, t = peaked_logits(w, rnd, DEV)
+        f = round_on(full, d, t)
+        parts = [round_on(halves[k], d[4 * k:4 * k + 4].contiguous(), t[4 * k:4 * k + 4].contiguous()) for k in range(2)]
+        for j in range(3):
+            assert torch.equal(f[j], torch.cat([parts[0][j], parts[1][j]]))
+    for hnd in [full] + halves:
+        hnd.destroy()
