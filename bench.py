@@ -1,0 +1,368 @@
+#!/usr/bin/env python
+"""Benchmark of the TapOut hot path: logit rows processed per second (draft + verify) on synthetic
+logits, with the HBM roofline of the dominant kernel and the CPU oracle timed beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one speculation round of the whole batch: k_max draft steps, verify, update.  Rows counted
+are those the method needs (draft rows of sequences still drafting, target rows up to the first
+rejection or the bonus row, and the draft row re-read for a residual).  Prints one JSON line (rank 0).
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2511_02017_b200 import synth_inputs as si  # noqa: E402
+
+METRIC = "logit rows processed/sec (draft+verify)"
+UNIT = "rows/s"
+POOL_ROUNDS = 3          # distinct pre-generated rounds cycled through (each far larger than L2)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index, period=0.004):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.stop_flag = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown",
+        }
+        while not self.stop_flag.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def result(self):
+        self.stop_flag.set()
+        if self.is_alive():
+            self.join(timeout=1.0)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def aggregate(rows_local, ms_local, world, backend_ready):
+    """Whole-job rows and the slowest rank's time.  No data-path collective exists; this is bookkeeping."""
+    if world == 1 or not backend_ready:
+        return rows_local, ms_local
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    r = torch.tensor([float(rows_local)], dtype=torch.float64, device=dev)
+    t = torch.tensor([float(ms_local)], dtype=torch.float64, device=dev)
+    dist.all_reduce(r, op=dist.ReduceOp.SUM)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(r.item()), float(t.item())
+
+
+# ----------------------------------------------------------------------------------------------
+def run_round(dev, w, draft, target, toks, cont, acc, nxt):
+    K = w.k_max
+    for i in range(K):
+        dev.draft_step(draft[:, i, :], toks[:, i], cont)
+    dev.verify(draft, target, toks, acc, nxt)
+    dev.update()
+
+
+def oracle_sample(w, draft, target, n_seq_sample, rounds, seq_offset=0):
+    """Times the oracle, as it stands, on `n_seq_sample` sequences of the given rounds' logits."""
+    from oracle import oracle as orc
+    from tests.lockstep import make_oracle
+    ids = np.arange(n_seq_sample)
+    ora = make_oracle(w, ids + seq_offset)
+    K = w.k_max
+    hosts = [(si.to_numpy_bits(d[:n_seq_sample]), si.to_numpy_bits(t[:n_seq_sample])) for d, t in zip(draft, target)]
+    t0 = time.perf_counter()
+    for r in range(rounds):
+        Dn, Tn = hosts[r % len(hosts)]
+        toks = np.full((n_seq_sample, K), -1, np.int32)
+        for i in range(K):
+            toks[:, i] = ora.draft_step(Dn[:, i, :])["token"]
+        ora.verify(Dn, Tn, toks)
+        ora.update()
+    dt = time.perf_counter() - t0
+    rows = ora.rows_read
+    cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    return rows, dt, cores
+
+
+def bench_ours(args):
+    from paper_2511_02017_b200 import binding as tp
+    rank, world, local = dist_env()
+    torch.cuda.set_device(local)
+    device = "cuda:%d" % local
+    backend_ready = False
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(device))
+        backend_ready = True
+    w = si.WORKLOADS[args.workload]
+    if args.n_seq:
+        w = si.scaled(w, n_seq=args.n_seq)          # profiling captures only: a smaller batch of the same rows
+    POOL_ROUNDS = args.pool_rounds
+    S, K, V = w.n_seq, w.k_max, w.vocab
+    # weak scaling: every rank owns a full-size shard of independent sequences, ids offset by rank
+    dev = tp.Tapout.from_workload(w, seq_offset=rank * S, token_out_stride=K)
+    if args.row_segments:
+        dev.set_param("row_segments", args.row_segments)
+    pool = [si.round_logits(si.scaled(w, seed=w.seed + 1000 * rank), r, device) for r in range(POOL_ROUNDS)]
+    toks = torch.full((S, K), -1, dtype=torch.int32, device=device)
+    cont = torch.empty(S, dtype=torch.uint8, device=device)
+    acc = torch.empty(S, dtype=torch.int32, device=device)
+    nxt = torch.empty(S, dtype=torch.int32, device=device)
+
+    def step(r):
+        d, t = pool[r % POOL_ROUNDS]
+        run_round(dev, w, d, t, toks, cont, acc, nxt)
+
+    for r in range(args.warmup):
+        step(r)
+    torch.cuda.synchronize()
+    st0 = dev.get_status()
+    l0 = dev.get_launch_count()
+    sampler = ClockSampler(physical_gpu_index(local))
+    if backend_ready:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for r in range(args.steps):
+        step(args.warmup + r)
+    e1.record()
+    torch.cuda.synchronize()
+    if backend_ready:
+        torch.distributed.barrier()
+    clocks = sampler.result()
+    ms = e0.elapsed_time(e1)
+    st1 = dev.get_status()
+    launches = dev.get_launch_count() - l0
+    rows_d = st1["rows_draft"] - st0["rows_draft"]
+    rows_t = st1["rows_target"] - st0["rows_target"]
+    rows_r = st1["rows_residual"] - st0["rows_residual"]
+    rows = rows_d + rows_t + rows_r
+    rows_all, ms_all = aggregate(rows, ms, world, backend_ready)
+    value = rows_all / (ms_all * 1e-3)
+
+    # ---- per-kernel device time (separate pass, same steps, events around the two streaming kernels)
+    dev.set_param("profile", 1)
+    dev.get_profile(0, reset=True)
+    dev.get_profile(1, reset=True)
+    sp0 = dev.get_status()
+    prof_steps = min(args.steps, 64)
+    for r in range(prof_steps):
+        step(args.warmup + args.steps + r)
+    torch.cuda.synchronize()
+    ms_rows, n_rows_l = dev.get_profile(0, reset=True)
+    ms_walk, n_walk_l = dev.get_profile(1, reset=True)
+    sp1 = dev.get_status()
+    dev.set_param("profile", 0)
+    peak, peak_src = measured_peaks()
+    row_bytes = w.row_bytes
+    b_rows = (sp1["rows_draft"] - sp0["rows_draft"]) * row_bytes
+    b_walk = ((sp1["rows_target"] - sp0["rows_target"]) + (sp1["rows_residual"] - sp0["rows_residual"])) * row_bytes
+    kernels = {
+        "k_draft_rows": {"launches": n_rows_l, "ms_total": ms_rows, "alg_bytes": b_rows,
+                         "gbs": b_rows / (ms_rows * 1e-3) / 1e9 if ms_rows > 0 else None},
+        "k_verify_walk": {"launches": n_walk_l, "ms_total": ms_walk, "alg_bytes": b_walk,
+                          "gbs": b_walk / (ms_walk * 1e-3) / 1e9 if ms_walk > 0 else None},
+    }
+    dom = max(kernels, key=lambda k: kernels[k]["ms_total"])
+    achieved = kernels[dom]["gbs"] or 0.0
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+                "alg_bytes_per_launch": kernels[dom]["alg_bytes"] / max(1, kernels[dom]["launches"]),
+                "avg_launch_ms": kernels[dom]["ms_total"] / max(1, kernels[dom]["launches"]),
+                "whole_step_gbs": rows * row_bytes / (ms * 1e-3) / 1e9,
+                "whole_step_frac_of_8TBs": rows * row_bytes / (ms * 1e-3) / 8e12}
+
+    # ---- end to end: host logits in pinned memory -> tapout_round_host -> host results
+    e2e = None
+    if not args.no_e2e:
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        hd, ht = pool[0][0].cpu().pin_memory(), pool[0][1].cpu().pin_memory()
+        o_tok = torch.empty((S, K), dtype=torch.int32).pin_memory()
+        o_acc = torch.empty(S, dtype=torch.int32).pin_memory()
+        o_nxt = torch.empty(S, dtype=torch.int32).pin_memory()
+        dev.set_param("token_out_stride", 1)
+        dev.round_host(hd, ht, o_tok, o_acc, o_nxt)                     # warm-up (allocates the staging buffers)
+        se0 = dev.get_status()
+        if backend_ready:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            dev.round_host(hd, ht, o_tok, o_acc, o_nxt)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        se1 = dev.get_status()
+        rows_e = sum(se1[k] - se0[k] for k in ("rows_draft", "rows_target", "rows_residual"))
+        rows_e_all, ms_e_all = aggregate(rows_e, dt * 1e3, world, backend_ready)
+        e2e = {"value": rows_e_all / (ms_e_all * 1e-3), "unit": UNIT, "steps": e2e_steps,
+               "ms_per_step": ms_e_all / e2e_steps,
+               "h2d_bytes_per_step": hd.numel() * hd.element_size() + ht.numel() * ht.element_size(),
+               "d2h_bytes_per_step": (o_tok.numel() + o_acc.numel() + o_nxt.numel()) * 4,
+               "api": "tapout_round_host (pinned host logits in, host tokens out)"}
+
+    # ---- CPU oracle on a bounded sample of the same workload (rank 0, single-GPU runs only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n_s = min(S, args.cpu_sample_seqs)
+        rows_o, dt_o, cores = oracle_sample(w, [pool[0][0]], [pool[0][1]], n_s, args.cpu_sample_rounds)
+        cpu = {"value": rows_o / dt_o, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": "%d of %d sequences, %d round(s) of this workload's logits, %d rows in %.1f s" %
+                         (n_s, S, args.cpu_sample_rounds, rows_o, dt_o)}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_all / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "%s: batch %d, vocab %d, %s logits, k_max %d, %s-level %s, %d arms" %
+                                   (w.name, S, V, w.dtype, K, w.level, w.policy, w.n_arms),
+                       "rows_per_step": rows / args.steps, "row_bytes": row_bytes,
+                       "l2_policy": "inputs larger than L2: %d rounds of %.2f GB cycled" %
+                                    (POOL_ROUNDS, (2 * K + 1) * S * row_bytes / 1e9),
+                       "sharding": "independent sequences per GPU, no collective" if world > 1 else "single GPU"},
+            "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "roofline": roofline, "kernels": kernels,
+            "rows": {"draft": rows_d, "target": rows_t, "residual": rows_r},
+            "hbm_gbs": rows * row_bytes / (ms * 1e-3) / 1e9,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    dev.destroy()
+    if backend_ready:
+        torch.distributed.destroy_process_group()
+
+
+def bench_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload."""
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    w = si.WORKLOADS[args.workload]
+    n_s = min(w.n_seq, args.ref_sample_seqs)
+    ws = si.scaled(w, n_seq=n_s)
+    pool = [si.round_logits(ws, r, "cpu") for r in range(2)]
+    K = w.k_max
+    for r in range(args.warmup):
+        oracle_sample(w, [pool[r % 2][0]], [pool[r % 2][1]], n_s, 1)
+    rows = 0
+    t0 = time.perf_counter()
+    cores = 1
+    for r in range(args.steps):
+        ro, _, cores = oracle_sample(w, [pool[r % 2][0]], [pool[r % 2][1]], n_s, 1)
+        rows += ro
+    dt = time.perf_counter() - t0
+    value = rows / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3 / max(1, args.steps), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s: batch %d, vocab %d, %s logits, k_max %d, %s-level %s, %d arms" %
+                               (w.name, w.n_seq, w.vocab, w.dtype, K, w.level, w.policy, w.n_arms),
+                   "sample": "each step = one round over %d of %d sequences" % (n_s, w.n_seq)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": "%d of %d sequences per step, %d steps" % (n_s, w.n_seq, args.steps)},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="throughput", choices=sorted(si.WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=6)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-seqs", type=int, default=256)
+    ap.add_argument("--cpu-sample-rounds", type=int, default=4)
+    ap.add_argument("--ref-sample-seqs", type=int, default=32)
+    ap.add_argument("--n-seq", type=int, default=0, help="override the batch size (profiling captures)")
+    ap.add_argument("--row-segments", type=int, default=0, help="CTAs per draft row (0 = library default)")
+    ap.add_argument("--pool-rounds", type=int, default=POOL_ROUNDS)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 20 if args.steps is None else args.steps
+        args.warmup = 2 if args.warmup is None else args.warmup
+        bench_reference(args)
+        return
+    args.steps = 400 if args.steps is None else args.steps
+    args.warmup = 8 if args.warmup is None else max(args.warmup, 3)
+    bench_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -125,6 +125,17 @@ class Tapout:
         for k, v in params.items():
             self.set_param(k, v)
 
+    @classmethod
+    def from_workload(cls, w, **params):
+        """Handle for a synth_inputs.Workload (its shapes, bandit, dtype, temperatures, seed), with the draft
+        tensor laid out [n_seq][k_max][vocab] so that step i reads column i."""
+        policy = {"ucb1": POLICY_UCB1, "ts": POLICY_TS, "ucb_tuned": POLICY_UCB_TUNED}[w.policy]
+        level = {"seq": LEVEL_SEQ, "token": LEVEL_TOKEN}[w.level]
+        return cls(w.n_seq, w.vocab, w.k_max, w.n_arms, policy, level, seed=w.seed,
+                   dtype=DTYPE_BF16 if w.dtype == "bf16" else DTYPE_FP32,
+                   inv_temp_draft=1.0 / w.temp_draft, inv_temp_target=1.0 / w.temp_target,
+                   step_row_stride=w.k_max * w.vocab, **params)
+
     def _check(self, rc, where):
         if rc != OK:
             detail = self.L.tapout_last_cuda_error(self.h).decode() if rc == E_CUDA else ""
