@@ -88,21 +88,13 @@ int setup_scratch(tapout* h) {
     Params& p = h->p;
     const int CH = chunk_of(h);
     p.NC = (p.V + CH - 1) / CH;
-    int nseg = h->nseg_user;
-    if (nseg <= 0) {
-        const long long want = 4LL * h->n_sm * 4;                 // about four waves of resident CTAs
-        nseg = (int)((want + p.S - 1) / p.S);
-        const int cap = p.NC / kWarps > 0 ? p.NC / kWarps : 1;    // keep every warp of a CTA busy
-        if (nseg > cap) nseg = cap;
-    }
-    if (nseg < 1) nseg = 1;
-    if (nseg > kMaxSeg) nseg = kMaxSeg;
-    if (nseg > p.NC) nseg = p.NC;
-    p.nseg = nseg;
+    p.nseg = h->nseg_user;                                   // 0: chosen on the device per launch
+    if (p.nseg > kMaxSeg) p.nseg = kMaxSeg;
+    if (p.nseg > p.NC) p.nseg = p.NC;
 
     if (h->d_scratch) { cudaFree(h->d_scratch); h->d_scratch = nullptr; }
     size_t off = 0;
-    const size_t o_seg = off;    off = align_up(off + sizeof(SegRec) * (size_t)p.S * p.nseg, 256);
+    const size_t o_seg = off;    off = align_up(off + sizeof(SegRec) * (size_t)p.S * kMaxSeg, 256);
     const size_t o_cdf = off;    off = align_up(off + sizeof(float2) * (size_t)p.S * p.NC, 256);
     const size_t o_list = off;   off = align_up(off + sizeof(int32_t) * 2 * (size_t)p.S, 256);
     const size_t o_count = off;  off = align_up(off + sizeof(int32_t) * 4, 256);
@@ -117,9 +109,7 @@ int setup_scratch(tapout* h) {
     h->sc.order = reinterpret_cast<int32_t*>(h->d_scratch + o_order);
     h->sc.status = reinterpret_cast<unsigned long long*>(h->d_scratch + o_status);
 
-    const long long items = (long long)p.S * p.nseg;
-    const long long res_rows = (long long)h->n_sm * 4;
-    h->grid_rows = (int)(items < res_rows ? items : res_rows);
+    h->grid_rows = h->n_sm * 3;                               // persistent: every CTA resident
     const long long res_walk = (long long)h->n_sm * 3;
     h->grid_walk = (int)(p.S < res_walk ? p.S : res_walk);
     return TAPOUT_OK;
@@ -169,18 +159,18 @@ int draft_step_impl(tapout* h, const void* logits, int64_t stride, int32_t* out_
     const float c = c_of(h->p.inv_Tq);
     { int rc = profile_mark(h, 0); if (rc) return rc; }
     if (h->p.dtype == DT_BF16)
-        k_draft_rows<DT_BF16><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->sc, logits, stride, parity, -1, c);
+        k_draft_rows<DT_BF16><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->sc, logits, stride, parity, -1, h->grid_rows, c);
     else
-        k_draft_rows<DT_FP32><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->sc, logits, stride, parity, -1, c);
+        k_draft_rows<DT_FP32><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->sc, logits, stride, parity, -1, h->grid_rows, c);
     TP_LAUNCHED(h);
     { int rc = profile_mark(h, 0); if (rc) return rc; }
     const int blocks = (h->p.S + 3) / 4;
     if (h->p.dtype == DT_BF16)
         k_draft_finish<DT_BF16><<<blocks, 128, 0, h->stream>>>(h->p, h->st, h->sc, logits, stride, h->pos, parity,
-                                                               h->round, c, out_token, tok_stride, out_continue);
+                                                               h->round, h->grid_rows, c, out_token, tok_stride, out_continue);
     else
         k_draft_finish<DT_FP32><<<blocks, 128, 0, h->stream>>>(h->p, h->st, h->sc, logits, stride, h->pos, parity,
-                                                               h->round, c, out_token, tok_stride, out_continue);
+                                                               h->round, h->grid_rows, c, out_token, tok_stride, out_continue);
     TP_LAUNCHED(h);
     h->pos += 1;
     return TAPOUT_OK;
@@ -195,7 +185,7 @@ int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const vo
         return TAPOUT_E_ALIGNMENT;
     k_verify_prepare<<<1, 1024, 0, h->stream>>>(h->p, h->st, h->sc);
     TP_LAUNCHED(h);
-    const size_t smem = sizeof(float2) * (size_t)h->p.NC;
+    const size_t smem = sizeof(double) * (size_t)chunk_of(h) + sizeof(float2) * (size_t)h->p.NC;
     const float cq = c_of(h->p.inv_Tq), cp = c_of(h->p.inv_Tp);
     { int rc = profile_mark(h, 1); if (rc) return rc; }
     if (h->p.dtype == DT_BF16)
@@ -504,14 +494,18 @@ int tapout_row_stats(tapout_t* h, const void* logits, int n_rows, int64_t row_st
     if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
     if (!aligned16(logits) || !stride_ok(h, row_stride) || row_stride < h->p.V) return TAPOUT_E_ALIGNMENT;
     const float c = c_of((float)inv_temp);
-    const long long items = (long long)n_rows * h->p.nseg;
-    const int grid = (int)(items < h->grid_rows ? items : h->grid_rows);
-    if (h->p.dtype == DT_BF16)
-        k_draft_rows<DT_BF16><<<grid, kThreads, 0, h->stream>>>(h->p, h->sc, logits, row_stride, 0, n_rows, c);
-    else
-        k_draft_rows<DT_FP32><<<grid, kThreads, 0, h->stream>>>(h->p, h->sc, logits, row_stride, 0, n_rows, c);
-    TP_LAUNCHED(h);
-    k_rows_features<<<(n_rows + 3) / 4, 128, 0, h->stream>>>(h->p, h->sc, n_rows, c, (float)inv_temp, out_features);
+    const int grid = h->grid_rows;
+    if (h->p.dtype == DT_BF16) {
+        k_draft_rows<DT_BF16><<<grid, kThreads, 0, h->stream>>>(h->p, h->sc, logits, row_stride, 0, n_rows, grid, c);
+        TP_LAUNCHED(h);
+        k_rows_features<DT_BF16><<<(n_rows + 3) / 4, 128, 0, h->stream>>>(h->p, h->sc, logits, row_stride, n_rows, grid, c,
+                                                                         (float)inv_temp, out_features);
+    } else {
+        k_draft_rows<DT_FP32><<<grid, kThreads, 0, h->stream>>>(h->p, h->sc, logits, row_stride, 0, n_rows, grid, c);
+        TP_LAUNCHED(h);
+        k_rows_features<DT_FP32><<<(n_rows + 3) / 4, 128, 0, h->stream>>>(h->p, h->sc, logits, row_stride, n_rows, grid, c,
+                                                                         (float)inv_temp, out_features);
+    }
     TP_LAUNCHED(h);
     return TAPOUT_OK;
 }

@@ -48,7 +48,7 @@ struct State {
 };
 
 // Partial result of one CTA over its share of a row.
-struct SegRec { float ref, S, T, m2; int argmax; int pad0, pad1, pad2; };
+struct SegRec { float ref, S, T, c2; int best; int pad0, pad1, pad2; };   // c2: second largest chunk maximum; best: lowest chunk holding ref
 
 struct Scratch {
     SegRec* seg;                 // [S][nseg]
@@ -328,25 +328,132 @@ __device__ __forceinline__ int cdf_locate(const float2* part, int NC, float c, d
     return pick;
 }
 
-// Token inside one chunk: weights recomputed in double, 32 tokens per step, token order.
-// WeightFn(idx) -> double weight of token idx (>= 0).  rem is in the same units.
-template <int CH, typename WeightFn>
-__device__ __forceinline__ int pick_in_chunk(int chunk, int V, double rem, int lane, WeightFn wf) {
-    const int base = chunk * CH;
-    double run = 0.0;
-    int last_pos = -1;
-    for (int i = 0; i < CH / 32; ++i) {
-        const int idx = base + i * 32 + lane;
-        if (base + i * 32 >= V) break;
-        const double w = (idx < V) ? wf(idx) : 0.0;
-        const unsigned posm = __ballot_sync(0xffffffffu, w > 0.0);
-        if (posm) last_pos = base + i * 32 + 31 - __clz(posm);
-        const double incl = warp_incl_scan_d(w, lane);
-        const unsigned over = __ballot_sync(0xffffffffu, run + incl > rem);
-        if (over) return base + i * 32 + __ffs(over) - 1;
-        run += __shfl_sync(0xffffffffu, incl, 31);
+// The lane's contiguous share of one chunk: EPL consecutive elements = 64 bytes = 4 raw vectors.
+// Vectors wholly at or beyond V are not read (zeros); lane_block_elem masks elements >= V to -inf.
+template <int DT>
+__device__ __forceinline__ void load_lane_block(const void* row, int V, int chunk, int lane, uint4 (&v)[4]) {
+    constexpr int PV = Elem<DT>::PV;
+    constexpr int EPL = chunk_elems<DT>() / 32;
+    const int e0 = chunk * chunk_elems<DT>() + lane * EPL;
+    const uint4* rp = reinterpret_cast<const uint4*>(row);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int e = e0 + j * PV;
+        v[j] = make_uint4(0, 0, 0, 0);
+        if (e < V) v[j] = __ldg(rp + e / PV);        // the row stride is a 16-byte multiple: in bounds
     }
-    return last_pos;
+}
+
+// Element k (0 <= k < EPL, compile-time after unrolling) of a lane block; idx = its token index.
+template <int DT>
+__device__ __forceinline__ float lane_block_elem(const uint4 (&v)[4], int k, int idx, int V) {
+    constexpr int PV = Elem<DT>::PV;
+    const uint4 q = v[k / PV];
+    const int r = k % PV;
+    float z;
+    if (DT == DT_BF16) {
+        const uint32_t w = (r / 2 == 0) ? q.x : (r / 2 == 1) ? q.y : (r / 2 == 2) ? q.z : q.w;
+        z = (r & 1) ? __uint_as_float(w & 0xffff0000u) : __uint_as_float(w << 16);
+    } else {
+        z = __uint_as_float(r == 0 ? q.x : r == 1 ? q.y : r == 2 ? q.z : q.w);
+    }
+    return idx < V ? z : neg_inf();
+}
+
+// Where the per-token weights of one chunk live while a token is picked: registers (finish kernel, one
+// warp per row, registers to spare) or shared memory (verify kernel, whose streaming loops set the budget).
+template <int EPL> struct RegWeights {
+    double w[EPL];
+    __device__ __forceinline__ void set(int k, double v) { w[k] = v; }
+    __device__ __forceinline__ double get(int k) const { return w[k]; }
+};
+template <int EPL> struct SmemWeights {
+    double* base;           // EPL * 32 doubles; element k of lane l at k*32 + l (conflict-free)
+    int lane;
+    __device__ __forceinline__ void set(int k, double v) { base[k * 32 + lane] = v; }
+    __device__ __forceinline__ double get(int k) const { return base[k * 32 + lane]; }
+};
+
+// Token inside one chunk.  Lane l owns the EPL consecutive tokens starting at first_token (its own);
+// W holds their weights in double (>= 0), rem is the target inside the chunk in the same units.  First
+// token whose running sum exceeds rem; if rounding leaves none, the last token with positive weight.
+template <int EPL, typename W>
+__device__ __forceinline__ int pick_in_block(const W& w, int first_token, double rem, int lane) {
+    double sum = 0.0;
+#pragma unroll
+    for (int k = 0; k < EPL; ++k) sum += w.get(k);
+    const double incl = warp_incl_scan_d(sum, lane);
+    const unsigned over = __ballot_sync(0xffffffffu, incl > rem);
+    const unsigned pos = __ballot_sync(0xffffffffu, sum > 0.0);
+    int L;
+    if (over) L = __ffs(over) - 1;
+    else if (pos) L = 31 - __clz(pos);
+    else return -1;
+    const double t = rem - (incl - sum);
+    double run = 0.0;
+    int pick = -1, last_pos = -1;
+    if (lane == L) {
+#pragma unroll
+        for (int k = 0; k < EPL; ++k) {
+            const double x = w.get(k);
+            if (x > 0.0) last_pos = k;
+            run += x;
+            if (pick < 0 && run > t) pick = k;
+        }
+        if (pick < 0) pick = last_pos;
+    }
+    return __shfl_sync(0xffffffffu, first_token + pick, L);
+}
+
+template <int DT, typename W>
+__device__ __forceinline__ int pick_softmax(W& w, const void* row, int V, int chunk, double rem, double inv_T,
+                                            double m_s, int lane) {
+    constexpr int EPL = chunk_elems<DT>() / 32;
+    const int e0 = chunk * chunk_elems<DT>() + lane * EPL;
+    uint4 v[4];
+    load_lane_block<DT>(row, V, chunk, lane, v);
+#pragma unroll
+    for (int k = 0; k < EPL; ++k) w.set(k, exp((double)lane_block_elem<DT>(v, k, e0 + k, V) * inv_T - m_s));
+    return pick_in_block<EPL>(w, e0, rem, lane);
+}
+
+template <int DT, typename W>
+__device__ __forceinline__ int pick_residual(W& w, const void* prow, const void* qrow, int V, int chunk, double rem,
+                                             double iTp, double lse_p, double iTq, double lse_q, int lane) {
+    constexpr int EPL = chunk_elems<DT>() / 32;
+    const int e0 = chunk * chunk_elems<DT>() + lane * EPL;
+    uint4 vp[4], vq[4];
+    load_lane_block<DT>(prow, V, chunk, lane, vp);
+    load_lane_block<DT>(qrow, V, chunk, lane, vq);
+#pragma unroll
+    for (int k = 0; k < EPL; ++k) {
+        const double r = exp((double)lane_block_elem<DT>(vp, k, e0 + k, V) * iTp - lse_p) -
+                         exp((double)lane_block_elem<DT>(vq, k, e0 + k, V) * iTq - lse_q);
+        w.set(k, r > 0.0 ? r : 0.0);
+    }
+    return pick_in_block<EPL>(w, e0, rem, lane);
+}
+
+// In one chunk: how many elements equal the row maximum m, the lowest index of one, and the largest
+// element below m.  Whole warp; every lane returns the same values.
+template <int DT>
+__device__ __forceinline__ void scan_top_chunk(const void* row, int V, int chunk, float m, int lane, int& cnt,
+                                               int& first, float& below) {
+    constexpr int EPL = chunk_elems<DT>() / 32;
+    uint4 v[4];
+    load_lane_block<DT>(row, V, chunk, lane, v);
+    int c = 0, f = 0x7fffffff;
+    float b = neg_inf();
+    const int e0 = chunk * chunk_elems<DT>() + lane * EPL;
+#pragma unroll
+    for (int k = 0; k < EPL; ++k) {
+        const float z = lane_block_elem<DT>(v, k, e0 + k, V);
+        if (z == m) { c += 1; f = min(f, e0 + k); }
+        else if (z < m) b = fmaxf(b, z);
+    }
+    cnt = __reduce_add_sync(0xffffffffu, c);
+    first = __reduce_min_sync(0xffffffffu, f);
+    below = warp_max_f(b);
 }
 
 // ------------------------------------------------------------------ bandits (double, one thread)

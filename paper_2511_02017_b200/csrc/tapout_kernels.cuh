@@ -8,42 +8,56 @@ namespace tpo {
 
 struct WarpRec { float ref, k, S, T, c1, c2; int best; int pad; };
 
+// How many CTAs share one draft row, decided on the device from the number of rows actually drafted at
+// this position (the host never learns it): enough items for about six per CTA, at least one chunk per
+// warp, at most kMaxSeg.  The streaming pass and its finish kernel must agree, hence one function.
+__device__ __forceinline__ int segments_for(const Params& p, int n_rows, int grid) {
+    if (p.nseg > 0) return p.nseg;
+    int nseg = (6 * grid + n_rows - 1) / max(n_rows, 1);
+    nseg = min(nseg, max(p.NC / kWarps, 1));
+    return max(1, min(nseg, min(kMaxSeg, p.NC)));
+}
+
 // ============================================================================================
 // Draft rows, streaming pass.  Work item = (sequence still drafting, segment of its row); a
 // persistent grid strides over the items.  Per item the CTA leaves a SegRec and, per 2 KB chunk,
-// the chunk's partial softmax sum (for the inverse-CDF draw in the finish kernel).
+// the chunk's partial softmax sum (for the inverse-CDF draw in the finish kernel).  Each warp keeps
+// the next chunk's loads in flight while it folds the current one.
 // ============================================================================================
 template <int DT>
-__global__ void __launch_bounds__(kThreads, 4)
+__global__ void __launch_bounds__(kThreads, 3)
 k_draft_rows(Params p, Scratch sc, const void* __restrict__ logits, long long row_stride, int parity,
-             int n_fixed, float c)
+             int n_fixed, int grid_ref, float c)
 {
-    constexpr int CH = chunk_elems<DT>();
     __shared__ WarpRec wrec[kWarps];
-    __shared__ float sh_C1, sh_C2;
-    __shared__ int sh_best, sh_cnt, sh_first, sh_below;
-
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_rows = (n_fixed >= 0) ? n_fixed : sc.count[parity];
     if (n_fixed < 0 && blockIdx.x == 0 && tid == 0) sc.count[parity ^ 1] = 0;   // this step's finish appends to it
     const int32_t* list = sc.list + (size_t)parity * p.S;
-    const int total = n_rows * p.nseg;
+    const int nseg = segments_for(p, n_rows, grid_ref);
+    const int total = n_rows * nseg;
 
     for (int item = blockIdx.x; item < total; item += gridDim.x) {
-        const int ai = item / p.nseg, g = item - ai * p.nseg;
+        const int ai = item / nseg, g = item - ai * nseg;
         const int s = (n_fixed >= 0) ? ai : list[ai];
         const char* row = reinterpret_cast<const char*>(logits) + (size_t)s * row_stride * Elem<DT>::BYTES;
-        const int c0 = (int)(((long long)g * p.NC) / p.nseg);
-        const int c1 = (int)(((long long)(g + 1) * p.NC) / p.nseg);
+        const int c0 = (int)(((long long)g * p.NC) / nseg);
+        const int c1 = (int)(((long long)(g + 1) * p.NC) / nseg);
         float2* part = sc.cdf + (size_t)s * p.NC;
 
         WarpAcc acc;
         acc.init();
-        for (int ch = c0 + warp; ch < c1; ch += kWarps) {
-            uint4 v[kVecPerLane];
-            load_chunk<DT>(row, p.V, ch, lane, v);
-            const float tot = fold_chunk<DT, true, true>(acc, v, ch, c);
+        int ch = c0 + warp;
+        uint4 cur[kVecPerLane], nxt[kVecPerLane];
+        if (ch < c1) load_chunk<DT>(row, p.V, ch, lane, cur);
+        while (ch < c1) {
+            const int chn = ch + kWarps;
+            if (chn < c1) load_chunk<DT>(row, p.V, chn, lane, nxt);
+            const float tot = fold_chunk<DT, true, true>(acc, cur, ch, c);
             if (lane == 0) part[ch] = make_float2(acc.ref, tot);
+#pragma unroll
+            for (int j = 0; j < kVecPerLane; ++j) cur[j] = nxt[j];
+            ch = chn;
         }
         const float Sw = warp_sum_f(acc.S), Tw = warp_sum_f(acc.T);
         if (lane == 0) {
@@ -52,81 +66,31 @@ k_draft_rows(Params p, Scratch sc, const void* __restrict__ logits, long long ro
             wrec[warp] = r;
         }
         __syncthreads();
-
-        float ref = neg_inf(), Sg = 0.f, Tg = 0.f;
-        if (tid == 0) {
-            // common reference = the largest of the warps' references; sums rescaled to it in double
-            float kref = 0.f;
-            bool any_nan = false;
-            for (int w = 0; w < kWarps; ++w) {
-                if (wrec[w].ref != wrec[w].ref) any_nan = true;
-                if (wrec[w].ref > ref) { ref = wrec[w].ref; kref = wrec[w].k; }
-            }
-            double Sd = 0.0, Td = 0.0;
-            for (int w = 0; w < kWarps; ++w) {
-                if (wrec[w].ref == neg_inf()) continue;
-                const double dd = (double)kref - (double)wrec[w].k;       // <= 0
-                const double f = exp2(dd);
-                Sd += f * (double)wrec[w].S;
-                Td += f * ((double)wrec[w].T + dd * (double)wrec[w].S);
-            }
-            Sg = (float)Sd; Tg = (float)Td;
-            if (any_nan) { Sg = __int_as_float(0x7fc00000); }
+        if (warp == 0) {
+            // lane w merges warp w's record: common reference = the largest, sums rescaled to it
+            WarpRec r;
+            r.ref = neg_inf(); r.k = 0.f; r.S = 0.f; r.T = 0.f; r.c1 = neg_inf(); r.c2 = neg_inf(); r.best = -1;
+            if (lane < kWarps) r = wrec[lane];
+            const bool live = r.ref != neg_inf();                 // a NaN reference counts as live and poisons S
+            const float ref = warp_max_f(r.ref);
+            const float kref = __fmul_rn(-ref, c);
+            const float dd = live ? kref - r.k : 0.f;             // <= 0
+            const float f = live ? ex2_approx(dd) : 0.f;
+            const float Sg = warp_sum_f(live ? f * r.S : 0.f);
+            const float Tg = warp_sum_f(live ? f * fmaf(dd, r.S, r.T) : 0.f);
             // two largest chunk maxima of the segment (with multiplicity); lowest chunk holding the largest
-            float C1 = neg_inf(), C2 = neg_inf();
-            int best = -1;
-            for (int w = 0; w < kWarps; ++w) {
-                const float a1 = wrec[w].c1, a2 = wrec[w].c2;
-                if (wrec[w].best < 0) continue;
-                if (a1 > C1) { C2 = C1; C1 = a1; best = wrec[w].best; }
-                else if (a1 == C1) { C2 = C1; best = min(best, wrec[w].best); }
-                else if (a1 > C2) { C2 = a1; }
-                if (a2 > C2) C2 = a2;          // a2 <= a1 <= C1 here
-            }
-            sh_C1 = C1; sh_C2 = C2; sh_best = best;
-            sh_cnt = 0; sh_first = 0x7fffffff; sh_below = (int)0x80000000;
-        }
-        __syncthreads();
-
-        // Second largest element and argmax: only the chunk holding the maximum needs a second look.
-        const int best = sh_best;
-        const float C1 = sh_C1;
-        if (best >= 0) {
-            int cnt = 0, first = 0x7fffffff;
-            float below = neg_inf();
-            for (int e = tid; e < CH; e += kThreads) {
-                const int idx = best * CH + e;
-                if (idx < p.V) {
-                    const float z = load_elem<DT>(row, idx);
-                    if (z == C1) { cnt += 1; first = min(first, idx); }
-                    else if (z < C1) below = fmaxf(below, z);
-                }
-            }
-            cnt = __reduce_add_sync(0xffffffffu, cnt);
-            first = __reduce_min_sync(0xffffffffu, first);
-            below = warp_max_f(below);
+            const unsigned tie = __ballot_sync(0xffffffffu, r.best >= 0 && r.c1 == ref);
+            const int win = tie ? __ffs(tie) - 1 : 0;
+            const float other = warp_max_f((lane == win) ? neg_inf() : r.c1);
+            const float c2all = warp_max_f(r.c2);
+            const float C2 = (__popc(tie) >= 2) ? ref : fmaxf(other, c2all);
+            const int best = __reduce_min_sync(0xffffffffu, (tie >> lane) & 1u ? r.best : 0x7fffffff);
             if (lane == 0) {
-                int bi = __float_as_int(below);
-                bi ^= (bi >> 31) & 0x7fffffff;
-                atomicAdd(&sh_cnt, cnt);
-                atomicMin(&sh_first, first);
-                atomicMax(&sh_below, bi);
+                SegRec o;
+                o.ref = ref; o.S = Sg; o.T = Tg; o.c2 = C2; o.best = (best == 0x7fffffff) ? -1 : best;
+                o.pad0 = o.pad1 = o.pad2 = 0;
+                sc.seg[(size_t)s * kMaxSeg + g] = o;
             }
-        }
-        __syncthreads();
-        if (tid == 0) {
-            SegRec r;
-            float m2 = sh_C2;
-            int am = -1;
-            if (best >= 0) {
-                int bi = sh_below;
-                bi ^= (bi >> 31) & 0x7fffffff;
-                const float within = (sh_cnt >= 2) ? C1 : __int_as_float(bi);
-                m2 = fmaxf(m2, within);
-                am = (sh_first == 0x7fffffff) ? -1 : sh_first;
-            }
-            r.ref = ref; r.S = Sg; r.T = Tg; r.m2 = m2; r.argmax = am; r.pad0 = r.pad1 = r.pad2 = 0;
-            sc.seg[(size_t)s * p.nseg + g] = r;
         }
         __syncthreads();
     }
@@ -142,23 +106,19 @@ struct RowComb {
     CdfTotals tot;
 };
 
-__device__ __forceinline__ RowComb combine_row(const Params& p, const Scratch& sc, int s, float c, int lane) {
+template <int DT>
+__device__ __forceinline__ RowComb combine_row(const Params& p, const Scratch& sc, const void* row, int s, int nseg,
+                                               float c, int lane) {
     RowComb rc;
     SegRec r;
-    r.ref = neg_inf(); r.S = 0.f; r.T = 0.f; r.m2 = neg_inf(); r.argmax = -1;
-    if (lane < p.nseg) r = sc.seg[(size_t)s * p.nseg + lane];
+    r.ref = neg_inf(); r.S = 0.f; r.T = 0.f; r.c2 = neg_inf(); r.best = -1;
+    if (lane < nseg) r = sc.seg[(size_t)s * kMaxSeg + lane];
     const bool has_nan = __any_sync(0xffffffffu, (r.S != r.S) || (r.T != r.T) || (r.ref != r.ref));
     const float m = warp_max_f(r.ref);
-    const unsigned tie = __ballot_sync(0xffffffffu, lane < p.nseg && r.ref == m);
-    const int win = tie ? __ffs(tie) - 1 : 0;
-    const float other = warp_max_f((lane == win || lane >= p.nseg) ? neg_inf() : r.ref);
-    const float m2all = warp_max_f(r.m2);
     rc.m = m;
-    rc.m2 = (__popc(tie) >= 2) ? m : fmaxf(other, m2all);
-    rc.argmax = __shfl_sync(0xffffffffu, r.argmax, win);
     rc.mc = (double)m * (double)c;
     double Tg = 0.0;
-    if (lane < p.nseg && r.ref > neg_inf() && r.ref < CUDART_INF_F) {
+    if (lane < nseg && r.ref > neg_inf() && r.ref < CUDART_INF_F) {
         const double d = (double)__fmul_rn(-r.ref, c) + rc.mc;           // >= 0 up to rounding
         Tg = exp2(-d) * ((double)r.T - d * (double)r.S);
     }
@@ -166,6 +126,21 @@ __device__ __forceinline__ RowComb combine_row(const Params& p, const Scratch& s
     rc.tot = cdf_totals(sc.cdf + (size_t)s * p.NC, p.NC, c, rc.mc, true, lane);
     rc.W = rc.tot.W;
     rc.valid = !has_nan && (m > neg_inf()) && (m < CUDART_INF_F) && (rc.W > 0.0) && (rc.W < CUDART_INF);
+    rc.m2 = neg_inf();
+    rc.argmax = -1;
+    if (rc.valid) {
+        // second largest element and argmax: only the (lowest) chunk holding the maximum needs a second look
+        const unsigned tie = __ballot_sync(0xffffffffu, lane < nseg && r.ref == m);
+        const int win = __ffs(tie) - 1;
+        const float other = warp_max_f((lane == win || lane >= nseg) ? neg_inf() : r.ref);
+        const float c2all = warp_max_f(r.c2);
+        const int best = __shfl_sync(0xffffffffu, r.best, win);
+        int cnt, first;
+        float below;
+        scan_top_chunk<DT>(row, p.V, best, m, lane, cnt, first, below);
+        rc.argmax = first;
+        rc.m2 = (__popc(tie) >= 2 || cnt >= 2) ? m : fmaxf(fmaxf(other, c2all), below);
+    }
     return rc;
 }
 
@@ -190,10 +165,9 @@ __device__ __forceinline__ RowFeat features_of(const RowComb& rc, float inv_T) {
 template <int DT>
 __global__ void __launch_bounds__(128)
 k_draft_finish(Params p, State st, Scratch sc, const void* __restrict__ logits, long long row_stride, int pos,
-               int parity, uint32_t round, float c, int32_t* __restrict__ out_token, long long tok_stride,
-               uint8_t* __restrict__ out_continue)
+               int parity, uint32_t round, int grid_ref, float c, int32_t* __restrict__ out_token,
+               long long tok_stride, uint8_t* __restrict__ out_continue)
 {
-    constexpr int CH = chunk_elems<DT>();
     __shared__ uint32_t hist[4][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int s = blockIdx.x * 4 + warp;
@@ -225,7 +199,9 @@ k_draft_finish(Params p, State st, Scratch sc, const void* __restrict__ logits, 
         else if (lane == 0) st.arm[(size_t)s * p.K + pos] = arm;
     }
 
-    const RowComb rc = combine_row(p, sc, s, c, lane);
+    const char* row = reinterpret_cast<const char*>(logits) + (size_t)s * row_stride * Elem<DT>::BYTES;
+    const int nseg = segments_for(p, sc.count[parity], grid_ref);
+    const RowComb rc = combine_row<DT>(p, sc, row, s, nseg, c, lane);
     if (lane == 0) atomicAdd(&sc.status[1], 1ull);
     if (!rc.valid) {
         if (lane == 0) {
@@ -237,14 +213,12 @@ k_draft_finish(Params p, State st, Scratch sc, const void* __restrict__ logits, 
     const RowFeat f = features_of(rc, p.inv_Tq);
 
     // ---- x_i ~ softmax(row): chunk by the partial sums, token inside the chunk in double
-    const char* row = reinterpret_cast<const char*>(logits) + (size_t)s * row_stride * Elem<DT>::BYTES;
     const uint4 w = rng_words(p, seq, round, (uint32_t)pos, RNG_DRAFT, 0, 0);
     const double u = u24_to_double(w.x);
     double rem;
     const int chunk = cdf_locate(sc.cdf + (size_t)s * p.NC, p.NC, c, rc.mc, true, lane, rc.tot, u * rc.W, rem);
-    const double inv_T = (double)p.inv_Tq, m_s = f.m_s;
-    const int tok = pick_in_chunk<CH>(chunk, p.V, rem, lane,
-                                      [&](int idx) { return exp((double)load_elem<DT>(row, idx) * inv_T - m_s); });
+    RegWeights<chunk_elems<DT>() / 32> wreg;
+    const int tok = pick_softmax<DT>(wreg, row, p.V, chunk, rem, (double)p.inv_Tq, f.m_s, lane);
 
     if (lane == 0) {
         float* fo = st.feat + ((size_t)s * p.K + pos) * kFeat;
@@ -266,13 +240,16 @@ k_draft_finish(Params p, State st, Scratch sc, const void* __restrict__ logits, 
 }
 
 // Features only (tapout_row_stats): one warp per row.
+template <int DT>
 __global__ void __launch_bounds__(128)
-k_rows_features(Params p, Scratch sc, int n_rows, float c, float inv_T, float* __restrict__ out)
+k_rows_features(Params p, Scratch sc, const void* __restrict__ logits, long long row_stride, int n_rows, int grid_ref,
+                float c, float inv_T, float* __restrict__ out)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int s = blockIdx.x * 4 + warp;
     if (s >= n_rows) return;
-    const RowComb rc = combine_row(p, sc, s, c, lane);
+    const char* row = reinterpret_cast<const char*>(logits) + (size_t)s * row_stride * Elem<DT>::BYTES;
+    const RowComb rc = combine_row<DT>(p, sc, row, s, segments_for(p, n_rows, grid_ref), c, lane);
     if (lane != 0) return;
     float* fo = out + (size_t)s * kFeat;
     if (!rc.valid) {
@@ -308,6 +285,23 @@ k_verify_prepare(Params p, State st, Scratch sc)
         const int slot = atomicAdd(&hist[st.n_drafted[s]], 1);
         sc.order[slot] = s;
     }
+}
+
+// Token picks of the verify kernel, kept out of line so that their double-precision exponentials do not
+// set the register budget of the streaming loops around them.
+template <int DT>
+__device__ __noinline__ int pick_softmax_smem(double* sm_w, const void* row, int V, int chunk, double rem,
+                                              double inv_T, double m_s, int lane) {
+    SmemWeights<chunk_elems<DT>() / 32> w{sm_w, lane};
+    return pick_softmax<DT>(w, row, V, chunk, rem, inv_T, m_s, lane);
+}
+
+template <int DT>
+__device__ __noinline__ int pick_residual_smem(double* sm_w, const void* prow, const void* qrow, int V, int chunk,
+                                               double rem, double iTp, double lse_p, double iTq, double lse_q,
+                                               int lane) {
+    SmemWeights<chunk_elems<DT>() / 32> w{sm_w, lane};
+    return pick_residual<DT>(w, prow, qrow, V, chunk, rem, iTp, lse_p, iTq, lse_q, lane);
 }
 
 // Softmax normaliser of one row by the whole CTA.  Every thread returns the raw maximum m and
@@ -354,9 +348,10 @@ k_verify_walk(Params p, State st, Scratch sc, const void* __restrict__ qlog, lon
               const void* __restrict__ plog, long long p_seq, long long p_pos, const int32_t* __restrict__ toks,
               uint32_t round, float cq, float cp, int32_t* __restrict__ out_acc, int32_t* __restrict__ out_next)
 {
-    constexpr int CH = chunk_elems<DT>();
     constexpr int ESZ = Elem<DT>::BYTES;
-    extern __shared__ float2 sm_part[];
+    extern __shared__ double sm_dyn[];                       // [chunk_elems] pick weights, then [NC] chunk partials
+    double* sm_w = sm_dyn;
+    float2* sm_part = reinterpret_cast<float2*>(sm_dyn + chunk_elems<DT>());
     __shared__ float2 wrec[kWarps];
     __shared__ int sh_i, sh_dec, sh_tok;
     __shared__ double sh_lse;
@@ -459,12 +454,8 @@ k_verify_walk(Params p, State st, Scratch sc, const void* __restrict__ qlog, lon
                 if (t.W > 0.0) {
                     double rem;
                     const int chunk = cdf_locate(sm_part, p.NC, 0.f, 0.0, false, lane, t, u2 * t.W, rem);
-                    const double iTp = (double)p.inv_Tp, iTq = (double)p.inv_Tq;
-                    tok = pick_in_chunk<CH>(chunk, p.V, rem * exp2(-dq), lane, [&](int idx) {
-                        const double r = exp((double)load_elem<DT>(prow, idx) * iTp - lse_p) -
-                                         exp((double)load_elem<DT>(qrow, idx) * iTq - lse_q);
-                        return r > 0.0 ? r : 0.0;
-                    });
+                    tok = pick_residual_smem<DT>(sm_w, prow, qrow, p.V, chunk, rem * exp2(-dq), (double)p.inv_Tp,
+                                                 lse_p, (double)p.inv_Tq, lse_q, lane);
                 }
                 if (lane == 0) sh_tok = tok;
             }
@@ -489,10 +480,8 @@ k_verify_walk(Params p, State st, Scratch sc, const void* __restrict__ qlog, lon
                     const CdfTotals t = cdf_totals(sm_part, p.NC, cp, mc, true, lane);
                     double rem;
                     const int chunk = cdf_locate(sm_part, p.NC, cp, mc, true, lane, t, u2 * t.W, rem);
-                    const double iTp = (double)p.inv_Tp, m_s = (double)m_p * iTp;
-                    const int tok = pick_in_chunk<CH>(chunk, p.V, rem, lane, [&](int idx) {
-                        return exp((double)load_elem<DT>(prow, idx) * iTp - m_s);
-                    });
+                    const int tok = pick_softmax_smem<DT>(sm_w, prow, p.V, chunk, rem, (double)p.inv_Tp,
+                                                          (double)m_p * (double)p.inv_Tp, lane);
                     if (lane == 0) sh_tok = tok;
                 }
                 __syncthreads();
