@@ -214,27 +214,28 @@ def bench_ours(args):
 
     # ---- per-kernel device time (separate pass, same steps, events around the two streaming kernels)
     dev.set_param("profile", 1)
-    dev.get_profile(0, reset=True)
-    dev.get_profile(1, reset=True)
+    for k in range(4):
+        dev.get_profile(k, reset=True)
     sp0 = dev.get_status()
     prof_steps = min(args.steps, 64)
     for r in range(prof_steps):
         step(args.warmup + args.steps + r)
     torch.cuda.synchronize()
-    ms_rows, n_rows_l = dev.get_profile(0, reset=True)
-    ms_walk, n_walk_l = dev.get_profile(1, reset=True)
+    prof = [dev.get_profile(k, reset=True) for k in range(4)]
     sp1 = dev.get_status()
     dev.set_param("profile", 0)
     peak, peak_src = measured_peaks()
     row_bytes = w.row_bytes
-    b_rows = (sp1["rows_draft"] - sp0["rows_draft"]) * row_bytes
-    b_walk = ((sp1["rows_target"] - sp0["rows_target"]) + (sp1["rows_residual"] - sp0["rows_residual"])) * row_bytes
-    kernels = {
-        "k_draft_rows": {"launches": n_rows_l, "ms_total": ms_rows, "alg_bytes": b_rows,
-                         "gbs": b_rows / (ms_rows * 1e-3) / 1e9 if ms_rows > 0 else None},
-        "k_verify_walk": {"launches": n_walk_l, "ms_total": ms_walk, "alg_bytes": b_walk,
-                          "gbs": b_walk / (ms_walk * 1e-3) / 1e9 if ms_walk > 0 else None},
-    }
+    d_rows = sp1["rows_draft"] - sp0["rows_draft"]
+    d0_rows = min(d_rows, prof_steps * S)                 # every sequence drafts at position 0
+    v_rows = (sp1["rows_target"] - sp0["rows_target"]) + (sp1["rows_residual"] - sp0["rows_residual"])
+
+    def kinfo(k, rows_k):
+        ms_k, n_k = prof[k]
+        return {"launches": n_k, "ms_total": ms_k, "alg_bytes": rows_k * row_bytes,
+                "gbs": rows_k * row_bytes / (ms_k * 1e-3) / 1e9 if ms_k > 0 else None}
+    kernels = {"k_draft_step@pos0": kinfo(0, d0_rows), "k_verify_walk": kinfo(1, v_rows),
+               "k_draft_step@pos>0": kinfo(2, d_rows - d0_rows), "k_update": kinfo(3, 0)}
     dom = max(kernels, key=lambda k: kernels[k]["ms_total"])
     achieved = kernels[dom]["gbs"] or 0.0
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",

@@ -103,8 +103,10 @@ typedef enum {
     TAPOUT_P_ROW_SEGMENTS = 30,    /* i64: CTAs that share one draft row (0 = chosen from n_seq)     */
     TAPOUT_P_TOKEN_OUT_STRIDE = 31,/* i64: elements between sequences in out_token of draft_step (default 1); with k_max the
                                       caller can aim step i at column i of its [n_seq][k_max] token matrix  */
-    TAPOUT_P_PROFILE = 32,         /* i64: 1 = time the two streaming kernels with CUDA events (tapout_get_profile) */
-    TAPOUT_P__COUNT = 33
+    TAPOUT_P_PROFILE = 32,         /* i64: 1 = time every kernel of the round with CUDA events (tapout_get_profile) */
+    TAPOUT_P_VERIFY_CLUSTER = 33,  /* i64: CTAs per thread-block cluster that walks one sequence in verify: 1, 2, 4, 8
+                                      (0 = chosen from vocab); reading it back gives the size in use      */
+    TAPOUT_P__COUNT = 34
 } tapout_param;
 
 /* Sticky status bits reported by tapout_get_status. */
@@ -241,10 +243,10 @@ int tapout_get_status(tapout_t* h, uint64_t* bits, uint64_t* rows_draft, uint64_
                       uint64_t* rows_residual);
 
 /*
- * With TAPOUT_P_PROFILE = 1 every launch of the two streaming kernels (0: draft row pass,
- * 1: verification walk) is bracketed by CUDA events on the handle's stream.  Synchronises,
- * returns the summed device time in milliseconds and the number of launches since the last
- * reset; reset != 0 clears both.
+ * With TAPOUT_P_PROFILE = 1 every kernel launch of the round is bracketed by CUDA events on the
+ * handle's stream, in four classes: 0 draft step at position 0, 1 verification walk, 2 draft steps at
+ * later positions, 3 update.  Synchronises, returns the summed device time in milliseconds and the
+ * number of launches of that class since the last reset; reset != 0 clears both.
  */
 int tapout_get_profile(tapout_t* h, int kernel, double* ms, uint64_t* launches, int reset);
 

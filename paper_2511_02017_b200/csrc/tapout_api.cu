@@ -22,6 +22,8 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace
 
+constexpr int kProf = 4;   // timed launch classes: draft step at position 0, verify, draft steps at later positions, update
+
 struct tapout {
     Params p{};
     int device = 0;
@@ -41,7 +43,10 @@ struct tapout {
     State st{};
     char* d_scratch = nullptr;
     Scratch sc{};
-    int grid_rows = 0, grid_walk = 0;
+    int grid_rows = 0;
+    int cluster_user = 0, cluster = 1;   // CTAs per verify cluster: requested (0 = automatic) and in use
+    size_t walk_smem = 0;
+    bool arms_ready = false;             // the arms of round `round` are chosen and the round's lists are set up
     // host-round staging
     char* d_stage = nullptr;
     size_t stage_bytes = 0;
@@ -50,9 +55,9 @@ struct tapout {
     int64_t tok_stride = 1;
     // optional event timing of the two streaming kernels
     bool profile = false;
-    std::vector<cudaEvent_t> ev[2];      // start/stop pairs not yet read back
-    double prof_ms[2] = {0.0, 0.0};
-    uint64_t prof_n[2] = {0, 0};
+    std::vector<cudaEvent_t> ev[kProf];  // start/stop pairs not yet read back
+    double prof_ms[kProf] = {};
+    uint64_t prof_n[kProf] = {};
 };
 
 namespace {
@@ -83,7 +88,30 @@ bool stride_ok(const tapout* h, int64_t stride_elems) { return stride_elems > 0 
 
 float c_of(float inv_T) { return (float)((double)inv_T * kLog2e); }
 
-// Scratch sizes depend on dtype (chunk length) and on the row split: (re)allocated when those change.
+// Largest power-of-two cluster (at most 8 CTAs, the portable limit) that still leaves every warp of a CTA
+// a chunk of its own per row.
+int auto_cluster(int NC) {
+    int cs = kMaxCluster;
+    while (cs > 1 && NC / cs < kWarps) cs >>= 1;
+    return cs;
+}
+
+template <typename Kernel>
+int cluster_fits(tapout* h, Kernel kernel, int cs, size_t smem) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)cs, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n;
+}
+
+// Scratch sizes depend on dtype (chunk length): (re)allocated when that changes.
 int setup_scratch(tapout* h) {
     Params& p = h->p;
     const int CH = chunk_of(h);
@@ -92,33 +120,58 @@ int setup_scratch(tapout* h) {
     if (p.nseg > kMaxSeg) p.nseg = kMaxSeg;
     if (p.nseg > p.NC) p.nseg = p.NC;
 
+    // verify clusters: the requested size, reduced until the device can co-schedule such a cluster
+    int cs = h->cluster_user > 0 ? h->cluster_user : auto_cluster(p.NC);
+    if (cs > p.NC) cs = 1;
+    for (;; cs >>= 1) {
+        h->walk_smem = sizeof(float2) * (size_t)((p.NC + cs - 1) / cs + 1);
+        if (h->walk_smem > 160 * 1024) return TAPOUT_E_UNSUPPORTED;      // vocabulary too large for the chunk table
+        const int fit = (p.dtype == DT_BF16) ? cluster_fits(h, k_verify_walk<DT_BF16>, cs, h->walk_smem)
+                                             : cluster_fits(h, k_verify_walk<DT_FP32>, cs, h->walk_smem);
+        if (fit > 0 || cs == 1) break;
+    }
+    h->cluster = cs;
+    TP_CUDA(h, cudaFuncSetAttribute(k_draft_step<DT_BF16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFeedSmem));
+    TP_CUDA(h, cudaFuncSetAttribute(k_draft_step<DT_FP32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFeedSmem));
+    TP_CUDA(h, cudaFuncSetAttribute(k_draft_step<DT_BF16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFeedSmem));
+    TP_CUDA(h, cudaFuncSetAttribute(k_draft_step<DT_FP32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFeedSmem));
+    if (h->walk_smem > 40 * 1024) {
+        TP_CUDA(h, cudaFuncSetAttribute(k_verify_walk<DT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
+        TP_CUDA(h, cudaFuncSetAttribute(k_verify_walk<DT_FP32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
+    }
+
     if (h->d_scratch) { cudaFree(h->d_scratch); h->d_scratch = nullptr; }
     size_t off = 0;
     const size_t o_seg = off;    off = align_up(off + sizeof(SegRec) * (size_t)p.S * kMaxSeg, 256);
     const size_t o_cdf = off;    off = align_up(off + sizeof(float2) * (size_t)p.S * p.NC, 256);
-    const size_t o_list = off;   off = align_up(off + sizeof(int32_t) * 2 * (size_t)p.S, 256);
+    const size_t o_list = off;   off = align_up(off + sizeof(int32_t) * 3 * (size_t)p.S, 256);
     const size_t o_count = off;  off = align_up(off + sizeof(int32_t) * 4, 256);
-    const size_t o_order = off;  off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
+    const size_t o_stop = off;   off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
+    const size_t o_next = off;   off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
+    const size_t o_done = off;   off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
     const size_t o_status = off; off = align_up(off + sizeof(unsigned long long) * 4, 256);
-    TP_CUDA(h, cudaMalloc(&h->d_scratch, off));
+    if (cudaMalloc(&h->d_scratch, off) != cudaSuccess) { cudaGetLastError(); return TAPOUT_E_ALLOC; }
     TP_CUDA(h, cudaMemsetAsync(h->d_scratch, 0, off, h->stream));
     h->sc.seg = reinterpret_cast<SegRec*>(h->d_scratch + o_seg);
     h->sc.cdf = reinterpret_cast<float2*>(h->d_scratch + o_cdf);
     h->sc.list = reinterpret_cast<int32_t*>(h->d_scratch + o_list);
     h->sc.count = reinterpret_cast<int32_t*>(h->d_scratch + o_count);
-    h->sc.order = reinterpret_cast<int32_t*>(h->d_scratch + o_order);
+    h->sc.stopped = reinterpret_cast<int32_t*>(h->d_scratch + o_stop);
+    h->sc.next_pos = reinterpret_cast<int32_t*>(h->d_scratch + o_next);
+    h->sc.done = reinterpret_cast<int32_t*>(h->d_scratch + o_done);
     h->sc.status = reinterpret_cast<unsigned long long*>(h->d_scratch + o_status);
 
     h->grid_rows = h->n_sm * 3;                               // persistent: every CTA resident
-    const long long res_walk = (long long)h->n_sm * 3;
-    h->grid_walk = (int)(p.S < res_walk ? p.S : res_walk);
+    h->arms_ready = false;
     return TAPOUT_OK;
 }
 
-int reset_round_state(tapout* h, int reset_adaedl) {
-    const int blocks = (h->p.S + 255) / 256;
-    k_reset_round<<<blocks, 256, 0, h->stream>>>(h->p, h->st, h->sc, reset_adaedl);
+// Chooses the arms of the coming round and sets up its lists; needed whenever no update ran since the
+// bandit statistics, the Philox inputs or the scratch memory last changed.
+int begin_round_now(tapout* h, int reset_adaedl) {
+    k_begin_round<<<(h->p.S + 3) / 4, 128, 0, h->stream>>>(h->p, h->st, h->sc, h->round, reset_adaedl);
     TP_LAUNCHED(h);
+    h->arms_ready = true;
     return TAPOUT_OK;
 }
 
@@ -150,30 +203,45 @@ int profile_mark(tapout* h, int k) {
     return TAPOUT_OK;
 }
 
+StepArgs step_args(const tapout* h, const void* logits, int64_t stride, float c) {
+    StepArgs a = {};
+    a.logits = logits; a.row_stride = stride;
+    a.pos = h->pos; a.slot = h->pos % 3; a.n_fixed = -1; a.grid_ref = h->grid_rows;
+    a.round = h->round; a.c = c; a.inv_T = h->p.inv_Tq;
+    a.tok_stride = 1;
+    return a;
+}
+
 int draft_step_impl(tapout* h, const void* logits, int64_t stride, int32_t* out_token, int64_t tok_stride,
                     uint8_t* out_continue) {
     if (!h || !logits || !out_token || !out_continue) return TAPOUT_E_INVALID_ARG;
     if (h->verified || h->pos >= h->p.K) return TAPOUT_E_BAD_STATE;
     if (!aligned16(logits) || !stride_ok(h, stride)) return TAPOUT_E_ALIGNMENT;
-    const int parity = h->pos & 1;
-    const float c = c_of(h->p.inv_Tq);
-    { int rc = profile_mark(h, 0); if (rc) return rc; }
-    if (h->p.dtype == DT_BF16)
-        k_draft_rows<DT_BF16><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->sc, logits, stride, parity, -1, h->grid_rows, c);
-    else
-        k_draft_rows<DT_FP32><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->sc, logits, stride, parity, -1, h->grid_rows, c);
+    if (h->pos == 0 && !h->arms_ready) { int rc = begin_round_now(h, 0); if (rc) return rc; }
+    StepArgs a = step_args(h, logits, stride, c_of(h->p.inv_Tq));
+    a.out_token = out_token; a.tok_stride = tok_stride; a.out_continue = out_continue;
+    const int pk = h->pos == 0 ? 0 : 2;
+    { int rc = profile_mark(h, pk); if (rc) return rc; }
+    if (h->p.dtype == DT_BF16) k_draft_step<DT_BF16, false><<<h->grid_rows, kStepThreads, kFeedSmem, h->stream>>>(h->p, h->st, h->sc, a);
+    else k_draft_step<DT_FP32, false><<<h->grid_rows, kStepThreads, kFeedSmem, h->stream>>>(h->p, h->st, h->sc, a);
     TP_LAUNCHED(h);
-    { int rc = profile_mark(h, 0); if (rc) return rc; }
-    const int blocks = (h->p.S + 3) / 4;
-    if (h->p.dtype == DT_BF16)
-        k_draft_finish<DT_BF16><<<blocks, 128, 0, h->stream>>>(h->p, h->st, h->sc, logits, stride, h->pos, parity,
-                                                               h->round, h->grid_rows, c, out_token, tok_stride, out_continue);
-    else
-        k_draft_finish<DT_FP32><<<blocks, 128, 0, h->stream>>>(h->p, h->st, h->sc, logits, stride, h->pos, parity,
-                                                               h->round, h->grid_rows, c, out_token, tok_stride, out_continue);
-    TP_LAUNCHED(h);
+    { int rc = profile_mark(h, pk); if (rc) return rc; }
     h->pos += 1;
     return TAPOUT_OK;
+}
+
+template <int DT>
+cudaError_t launch_walk(tapout* h, const WalkArgs& a) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)h->p.S * (unsigned)h->cluster, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = h->walk_smem;
+    cfg.stream = h->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)h->cluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_verify_walk<DT>, h->p, h->st, h->sc, a);
 }
 
 int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const void* pl, int64_t p_seq, int64_t p_pos,
@@ -183,17 +251,13 @@ int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const vo
     if (!aligned16(q) || !aligned16(pl) || !stride_ok(h, q_seq) || !stride_ok(h, q_pos) || !stride_ok(h, p_seq) ||
         !stride_ok(h, p_pos))
         return TAPOUT_E_ALIGNMENT;
-    k_verify_prepare<<<1, 1024, 0, h->stream>>>(h->p, h->st, h->sc);
-    TP_LAUNCHED(h);
-    const size_t smem = sizeof(double) * (size_t)chunk_of(h) + sizeof(float2) * (size_t)h->p.NC;
-    const float cq = c_of(h->p.inv_Tq), cp = c_of(h->p.inv_Tp);
+    WalkArgs a = {};
+    a.qlog = q; a.q_seq = q_seq; a.q_pos = q_pos; a.plog = pl; a.p_seq = p_seq; a.p_pos = p_pos;
+    a.toks = toks; a.slot = h->pos % 3; a.round = h->round;
+    a.cq = c_of(h->p.inv_Tq); a.cp = c_of(h->p.inv_Tp);
+    a.out_acc = out_acc; a.out_next = out_next;
     { int rc = profile_mark(h, 1); if (rc) return rc; }
-    if (h->p.dtype == DT_BF16)
-        k_verify_walk<DT_BF16><<<h->grid_walk, kThreads, smem, h->stream>>>(h->p, h->st, h->sc, q, q_seq, q_pos, pl, p_seq,
-                                                                          p_pos, toks, h->round, cq, cp, out_acc, out_next);
-    else
-        k_verify_walk<DT_FP32><<<h->grid_walk, kThreads, smem, h->stream>>>(h->p, h->st, h->sc, q, q_seq, q_pos, pl, p_seq,
-                                                                          p_pos, toks, h->round, cq, cp, out_acc, out_next);
+    TP_CUDA(h, h->p.dtype == DT_BF16 ? launch_walk<DT_BF16>(h, a) : launch_walk<DT_FP32>(h, a));
     TP_LAUNCHED(h);
     { int rc = profile_mark(h, 1); if (rc) return rc; }
     h->verified = true;
@@ -203,11 +267,14 @@ int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const vo
 int update_impl(tapout* h) {
     if (!h) return TAPOUT_E_INVALID_ARG;
     if (!h->verified) return TAPOUT_E_BAD_STATE;
-    k_update<<<(h->p.S + 255) / 256, 256, 0, h->stream>>>(h->p, h->st, h->sc);
+    { int rc = profile_mark(h, 3); if (rc) return rc; }
+    k_update<<<(h->p.S + 3) / 4, 128, 0, h->stream>>>(h->p, h->st, h->sc, h->round + 1);
     TP_LAUNCHED(h);
+    { int rc = profile_mark(h, 3); if (rc) return rc; }
     h->round += 1;
     h->pos = 0;
     h->verified = false;
+    h->arms_ready = true;
     return TAPOUT_OK;
 }
 
@@ -278,7 +345,7 @@ int tapout_create(tapout_t** out, int n_seq, int vocab, int k_max, int n_arms, i
     h->st.reward = (double*)at(12);
 
     int rc = setup_scratch(h);
-    if (rc == TAPOUT_OK) rc = reset_round_state(h, 1);
+    if (rc == TAPOUT_OK) rc = begin_round_now(h, 1);
     if (rc != TAPOUT_OK) { tapout_destroy(h); return rc == TAPOUT_E_CUDA ? TAPOUT_E_ALLOC : rc; }
     *out = h;
     return TAPOUT_OK;
@@ -287,7 +354,7 @@ int tapout_create(tapout_t** out, int n_seq, int vocab, int k_max, int n_arms, i
 int tapout_destroy(tapout_t* h) {
     if (!h) return TAPOUT_E_INVALID_ARG;
     cudaStreamSynchronize(h->stream);
-    for (int k = 0; k < 2; ++k) { for (cudaEvent_t e : h->ev[k]) cudaEventDestroy(e); h->ev[k].clear(); }
+    for (int k = 0; k < kProf; ++k) { for (cudaEvent_t e : h->ev[k]) cudaEventDestroy(e); h->ev[k].clear(); }
     if (h->d_state) cudaFree(h->d_state);
     if (h->d_scratch) cudaFree(h->d_scratch);
     if (h->d_stage) cudaFree(h->d_stage);
@@ -307,6 +374,7 @@ int tapout_set_param_i64(tapout_t* h, int key, int64_t v) {
     if (!h) return TAPOUT_E_INVALID_ARG;
     if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
     Params& p = h->p;
+    h->arms_ready = false;                 // the arm choice may depend on what changes here
     switch (key) {
     case TAPOUT_P_SEED: h->seed = (uint64_t)v; p.seed_lo = (uint32_t)h->seed; p.seed_hi = (uint32_t)(h->seed >> 32); return TAPOUT_OK;
     case TAPOUT_P_DTYPE:
@@ -316,7 +384,7 @@ int tapout_set_param_i64(tapout_t* h, int key, int64_t v) {
             TP_CUDA(h, cudaStreamSynchronize(h->stream));
             int rc = setup_scratch(h);
             if (rc != TAPOUT_OK) return rc;
-            return reset_round_state(h, 0);
+            return begin_round_now(h, 0);
         }
         return TAPOUT_OK;
     case TAPOUT_P_SEQ_OFFSET: if (v < 0 || v > 0xffffffffLL) return TAPOUT_E_INVALID_ARG; p.seq_offset = (uint32_t)v; return TAPOUT_OK;
@@ -337,7 +405,15 @@ int tapout_set_param_i64(tapout_t* h, int key, int64_t v) {
         TP_CUDA(h, cudaStreamSynchronize(h->stream));
         int rc = setup_scratch(h);
         if (rc != TAPOUT_OK) return rc;
-        return reset_round_state(h, 0);
+        return begin_round_now(h, 0);
+    }
+    case TAPOUT_P_VERIFY_CLUSTER: {
+        if (v != 0 && v != 1 && v != 2 && v != 4 && v != 8) return TAPOUT_E_INVALID_ARG;
+        h->cluster_user = (int)v;
+        TP_CUDA(h, cudaStreamSynchronize(h->stream));
+        int rc = setup_scratch(h);
+        if (rc != TAPOUT_OK) return rc;
+        return begin_round_now(h, 0);
     }
     default: return TAPOUT_E_INVALID_ARG;
     }
@@ -348,6 +424,7 @@ int tapout_set_param_f64(tapout_t* h, int key, double v) {
     if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
     if (v != v) return TAPOUT_E_INVALID_ARG;
     Params& p = h->p;
+    h->arms_ready = false;
     switch (key) {
     case TAPOUT_P_INV_TEMP_DRAFT: if (!(v > 0.0) || !((float)v < 1e30f)) return TAPOUT_E_INVALID_ARG; p.inv_Tq = (float)v; return TAPOUT_OK;
     case TAPOUT_P_INV_TEMP_TARGET: if (!(v > 0.0) || !((float)v < 1e30f)) return TAPOUT_E_INVALID_ARG; p.inv_Tp = (float)v; return TAPOUT_OK;
@@ -360,8 +437,8 @@ int tapout_set_param_f64(tapout_t* h, int key, double v) {
     case TAPOUT_P_ADA_BETA1: p.ada_beta1 = v; return TAPOUT_OK;
     case TAPOUT_P_ADA_BETA2: p.ada_beta2 = v; return TAPOUT_OK;
     case TAPOUT_P_ADA_EPS: p.ada_eps = v; return TAPOUT_OK;
-    case TAPOUT_P_ADA_LAMBDA0: p.ada_lambda0 = v; return reset_round_state(h, 1);
-    case TAPOUT_P_ADA_ACC0: p.ada_acc0 = v; return reset_round_state(h, 1);
+    case TAPOUT_P_ADA_LAMBDA0: p.ada_lambda0 = v; return begin_round_now(h, 1);
+    case TAPOUT_P_ADA_ACC0: p.ada_acc0 = v; return begin_round_now(h, 1);
     case TAPOUT_P_REWARD_ALPHA: p.reward_alpha = v; return TAPOUT_OK;
     case TAPOUT_P_UCB_C2: if (v < 0.0) return TAPOUT_E_INVALID_ARG; p.ucb_c2 = v; return TAPOUT_OK;
     case TAPOUT_P_TS_MU0: p.ts_mu0 = v; return TAPOUT_OK;
@@ -388,6 +465,7 @@ int tapout_get_param_i64(const tapout_t* h, int key, int64_t* v) {
     case TAPOUT_P_TS_BETA_B0: *v = p.ts_b0; return TAPOUT_OK;
     case TAPOUT_P_TOKEN_UPDATE_ALL: *v = p.token_update_all; return TAPOUT_OK;
     case TAPOUT_P_ROW_SEGMENTS: *v = p.nseg; return TAPOUT_OK;
+    case TAPOUT_P_VERIFY_CLUSTER: *v = h->cluster; return TAPOUT_OK;
     case TAPOUT_P_TOKEN_OUT_STRIDE: *v = h->tok_stride; return TAPOUT_OK;
     case TAPOUT_P_PROFILE: *v = h->profile ? 1 : 0; return TAPOUT_OK;
     default: return TAPOUT_E_INVALID_ARG;
@@ -426,6 +504,7 @@ int tapout_set_arms(tapout_t* h, const int32_t* rule_ids, int n) {
     for (int a = 0; a < n; ++a)
         if (rule_ids[a] < 0 || rule_ids[a] > TAPOUT_RULE_STATIC) return TAPOUT_E_INVALID_ARG;
     for (int a = 0; a < n; ++a) h->p.rule_of_arm[a] = rule_ids[a];
+    h->arms_ready = false;
     return TAPOUT_OK;
 }
 
@@ -493,19 +572,10 @@ int tapout_row_stats(tapout_t* h, const void* logits, int n_rows, int64_t row_st
     if (!(inv_temp > 0.0)) return TAPOUT_E_INVALID_ARG;
     if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
     if (!aligned16(logits) || !stride_ok(h, row_stride) || row_stride < h->p.V) return TAPOUT_E_ALIGNMENT;
-    const float c = c_of((float)inv_temp);
-    const int grid = h->grid_rows;
-    if (h->p.dtype == DT_BF16) {
-        k_draft_rows<DT_BF16><<<grid, kThreads, 0, h->stream>>>(h->p, h->sc, logits, row_stride, 0, n_rows, grid, c);
-        TP_LAUNCHED(h);
-        k_rows_features<DT_BF16><<<(n_rows + 3) / 4, 128, 0, h->stream>>>(h->p, h->sc, logits, row_stride, n_rows, grid, c,
-                                                                         (float)inv_temp, out_features);
-    } else {
-        k_draft_rows<DT_FP32><<<grid, kThreads, 0, h->stream>>>(h->p, h->sc, logits, row_stride, 0, n_rows, grid, c);
-        TP_LAUNCHED(h);
-        k_rows_features<DT_FP32><<<(n_rows + 3) / 4, 128, 0, h->stream>>>(h->p, h->sc, logits, row_stride, n_rows, grid, c,
-                                                                         (float)inv_temp, out_features);
-    }
+    StepArgs a = step_args(h, logits, row_stride, c_of((float)inv_temp));
+    a.n_fixed = n_rows; a.inv_T = (float)inv_temp; a.out_feat = out_features;
+    if (h->p.dtype == DT_BF16) k_draft_step<DT_BF16, true><<<h->grid_rows, kStepThreads, kFeedSmem, h->stream>>>(h->p, h->st, h->sc, a);
+    else k_draft_step<DT_FP32, true><<<h->grid_rows, kStepThreads, kFeedSmem, h->stream>>>(h->p, h->st, h->sc, a);
     TP_LAUNCHED(h);
     return TAPOUT_OK;
 }
@@ -537,8 +607,10 @@ int tapout_get_state(tapout_t* h, void* host_dst) {
 int tapout_set_state(tapout_t* h, const void* host_src) {
     if (!h || !host_src) return TAPOUT_E_INVALID_ARG;
     TP_CUDA(h, cudaMemcpyAsync(h->d_state, host_src, h->state_bytes, cudaMemcpyHostToDevice, h->stream));
-    if (!h->verified && h->pos < h->p.K) {
-        k_rebuild_active<<<1, 1024, 0, h->stream>>>(h->p, h->st, h->sc, h->pos & 1);
+    if (between_rounds(h)) {
+        h->arms_ready = false;             // statistics changed: the coming round's arms are chosen afresh
+    } else if (!h->verified) {
+        k_rebuild_lists<<<1, 1024, 0, h->stream>>>(h->p, h->st, h->sc, h->pos);
         TP_LAUNCHED(h);
     }
     TP_CUDA(h, cudaStreamSynchronize(h->stream));
@@ -556,6 +628,7 @@ int tapout_set_round(tapout_t* h, uint32_t round) {
     if (!h) return TAPOUT_E_INVALID_ARG;
     if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
     h->round = round;
+    h->arms_ready = false;
     return TAPOUT_OK;
 }
 
@@ -572,7 +645,7 @@ int tapout_get_status(tapout_t* h, uint64_t* bits, uint64_t* rows_draft, uint64_
 }
 
 int tapout_get_profile(tapout_t* h, int kernel, double* ms, uint64_t* launches, int reset) {
-    if (!h || kernel < 0 || kernel > 1) return TAPOUT_E_INVALID_ARG;
+    if (!h || kernel < 0 || kernel >= kProf) return TAPOUT_E_INVALID_ARG;
     if (h->ev[kernel].size() % 2 != 0) return TAPOUT_E_BAD_STATE;
     int rc = drain_profile(h, kernel);
     if (rc != TAPOUT_OK) return rc;

@@ -51,11 +51,13 @@ struct State {
 struct SegRec { float ref, S, T, c2; int best; int pad0, pad1, pad2; };   // c2: second largest chunk maximum; best: lowest chunk holding ref
 
 struct Scratch {
-    SegRec* seg;                 // [S][nseg]
+    SegRec* seg;                 // [S][kMaxSeg]
     float2* cdf;                 // [S][NC]: (reference logit, sum of 2^(z*c + k)) per chunk
-    int32_t* list;               // [2][S] sequences still drafting, ping-pong by position parity
-    int32_t* count;              // [0],[1] lengths of the two lists; [2] verify queue head
-    int32_t* order;              // [S] verify order, longest drafts first
+    int32_t* list;               // [3][S] sequences drafting at position pos, in slot pos % 3
+    int32_t* count;              // [0..2] lengths of the three lists; [3] length of `stopped`
+    int32_t* stopped;            // [S] sequences in the order in which they stopped drafting this round
+    int32_t* next_pos;           // [S] position the sequence drafts at next (stays put once it has stopped)
+    int32_t* done;               // [S] segments of the sequence's current row already reduced
     unsigned long long* status;  // [0] sticky bits, [1] draft rows, [2] target rows, [3] residual rows
 };
 
@@ -168,6 +170,216 @@ __device__ __forceinline__ void load_chunk(const void* row, int V, int ch, int l
     }
 }
 
+// ------------------------------------------------------------------ asynchronous chunk pipeline
+// Each warp keeps kDepth full 2 KB chunks on their way from global to its own ring in shared memory:
+// one lane issues a bulk asynchronous copy per chunk (the TMA unit moves the bytes, no registers are
+// held), completion is signalled on an mbarrier of the warp's own.  A chunk that reaches past the end of
+// the row is not copied this way: it is read with plain loads.  Every wait is bounded; if one gives up
+// the warp records it in the status word and reads this and all later chunks with plain loads.
+constexpr int kDepth = 4;
+constexpr int kChunkBytes = 32 * kVecPerLane * 16;
+constexpr int kRingBytes = kWarps * kDepth * kChunkBytes;       // per CTA
+constexpr int kPipeSmem = kRingBytes + kWarps * kDepth * 8;     // ring + mbarriers
+constexpr int kWaitTries = 1 << 22;
+constexpr unsigned long long kStCopyTimeout = 16ull;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+template <int DT> __device__ __forceinline__ bool chunk_is_full(int V, int ch) { return (ch + 1) * chunk_elems<DT>() <= V; }
+
+struct WarpPipe {
+    uint32_t data, bars;          // shared-space addresses of this warp's ring and of its kDepth mbarriers
+    uint32_t issued, taken;       // full chunks issued / taken so far
+    bool broken;
+
+    // ring: kRingBytes, 128-byte aligned; bar: kWarps * kDepth words of 8 bytes.  Call once per kernel, all lanes.
+    __device__ __forceinline__ void init(unsigned char* ring, unsigned long long* bar, int warp, int lane) {
+        data = smem_u32(ring) + (uint32_t)warp * kDepth * kChunkBytes;
+        bars = smem_u32(bar) + (uint32_t)warp * kDepth * 8;
+        issued = taken = 0;
+        broken = false;
+        if (lane == 0) {
+#pragma unroll
+            for (int d = 0; d < kDepth; ++d) mbar_init(bars + 8 * d, 1);
+            fence_proxy_async();
+        }
+        __syncwarp();
+    }
+    __device__ __forceinline__ int in_flight() const { return (int)(issued - taken); }
+    // src: 16-byte aligned start of a full chunk.  Needs in_flight() < kDepth.
+    __device__ __forceinline__ void issue(const void* src, int lane) {
+        if (broken) return;
+        __syncwarp();                                  // every lane has read the stage that is overwritten now
+        const uint32_t st = issued % kDepth;
+        if (lane == 0) {
+            fence_proxy_async();
+            mbar_expect_tx(bars + 8 * st, kChunkBytes);
+            bulk_g2s(data + st * kChunkBytes, src, kChunkBytes, bars + 8 * st);
+        }
+        issued += 1;
+    }
+    __device__ __forceinline__ bool wait_stage(uint32_t k) const {
+        const uint32_t bar = bars + 8 * (k % kDepth), parity = (k / kDepth) & 1u;
+        bool ok = false;
+        for (int it = 0; it < kWaitTries && !ok; ++it) ok = mbar_try_wait(bar, parity);
+        return __all_sync(0xffffffffu, ok);
+    }
+    // The oldest chunk in flight, in the lane layout of load_chunk.  row / ch name the same chunk for the
+    // fallback path.
+    template <int DT>
+    __device__ __forceinline__ void take(const void* row, int V, int ch, int lane, uint4 (&v)[kVecPerLane],
+                                         unsigned long long* status) {
+        if (!broken) {
+            if (wait_stage(taken)) {
+                const uint32_t base = data + (taken % kDepth) * kChunkBytes + (uint32_t)lane * 16;
+#pragma unroll
+                for (int j = 0; j < kVecPerLane; ++j) v[j] = lds128(base + j * 512);
+                taken += 1;
+                return;
+            }
+            broken = true;
+            if (lane == 0) atomicOr(status, kStCopyTimeout);
+        }
+        load_chunk<DT>(row, V, ch, lane, v);
+    }
+    // Before the CTA exits after a wait gave up: its copies still in flight are given a second bounded wait.
+    __device__ __forceinline__ void drain() const {
+        if (!broken) return;
+        for (uint32_t k = taken; k != issued; ++k) wait_stage(k);
+    }
+};
+
+// ---- the same ring fed by a producer: one extra warp per CTA issues the copies (lane w feeds the ring
+// of folding warp w and runs ahead of it by up to kDepth chunks, across work items), the folding warps
+// only wait, read and hand the stage back.  full[w][d]: copy landed (1 arrival + 2048 bytes);
+// empty[w][d]: all 32 lanes of warp w have read the stage.
+constexpr int kFeedSmem = kRingBytes + 2 * kWarps * kDepth * 8 + 64;     // ring, full, empty, issued counts, flag
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+struct FeedLayout {
+    unsigned char* ring;
+    unsigned long long* full;
+    unsigned long long* empty;
+    uint32_t* issued;            // [kWarps] chunks each producer lane has issued, written when it is done
+    uint32_t* flag;              // nonzero once any wait gave up
+    __device__ __forceinline__ explicit FeedLayout(unsigned char* base) {
+        ring = base;
+        full = reinterpret_cast<unsigned long long*>(base + kRingBytes);
+        empty = full + kWarps * kDepth;
+        issued = reinterpret_cast<uint32_t*>(empty + kWarps * kDepth);
+        flag = issued + kWarps;
+    }
+    // All threads of the CTA; followed by a CTA-wide barrier at the caller.
+    __device__ __forceinline__ void init(int tid) const {
+        if (tid < kWarps * kDepth) {
+            mbar_init(smem_u32(full + tid), 1);
+            mbar_init(smem_u32(empty + tid), 32);
+        }
+        if (tid < kWarps) issued[tid] = 0;
+        if (tid == 0) *flag = 0;
+        fence_proxy_async();
+    }
+};
+
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    bool ok = false;
+    for (int it = 0; it < kWaitTries && !ok; ++it) ok = mbar_try_wait(bar, parity);
+    return ok;
+}
+
+// One lane of the producer warp.
+struct FeedProducer {
+    uint32_t data, full, empty, n;
+    bool dead;
+    __device__ __forceinline__ void init(const FeedLayout& L, int w) {
+        data = smem_u32(L.ring) + (uint32_t)w * kDepth * kChunkBytes;
+        full = smem_u32(L.full + w * kDepth);
+        empty = smem_u32(L.empty + w * kDepth);
+        n = 0;
+        dead = false;
+    }
+    // src: 16-byte aligned start of a full chunk.  Waits until the stage it goes to has been read.
+    __device__ __forceinline__ void issue(const void* src, const FeedLayout& L, unsigned long long* status) {
+        if (dead) return;
+        const uint32_t st = n % kDepth;
+        if (n >= kDepth && !mbar_wait_bounded(empty + 8 * st, ((n / kDepth) - 1u) & 1u)) {
+            dead = true;
+            atomicOr(status, kStCopyTimeout);
+            atomicOr(L.flag, 1u);
+            return;
+        }
+        mbar_expect_tx(full + 8 * st, kChunkBytes);
+        bulk_g2s(data + st * kChunkBytes, src, kChunkBytes, full + 8 * st);
+        n += 1;
+    }
+};
+
+// A folding warp (all 32 lanes).
+struct FeedConsumer {
+    uint32_t data, full, empty, taken;
+    bool broken;
+    __device__ __forceinline__ void init(const FeedLayout& L, int w) {
+        data = smem_u32(L.ring) + (uint32_t)w * kDepth * kChunkBytes;
+        full = smem_u32(L.full + w * kDepth);
+        empty = smem_u32(L.empty + w * kDepth);
+        taken = 0;
+        broken = false;
+    }
+    // The warp's next full chunk, in the lane layout of load_chunk.  row / ch name the same chunk for the
+    // plain-load path that takes over once a wait has given up.
+    template <int DT>
+    __device__ __forceinline__ void take(const void* row, int V, int ch, int lane, uint4 (&v)[kVecPerLane],
+                                         const FeedLayout& L, unsigned long long* status) {
+        if (!broken) {
+            const uint32_t st = taken % kDepth;
+            const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(full + 8 * st, (taken / kDepth) & 1u));
+            if (ok) {
+                const uint32_t base = data + st * kChunkBytes + (uint32_t)lane * 16;
+#pragma unroll
+                for (int j = 0; j < kVecPerLane; ++j) v[j] = lds128(base + j * 512);
+                mbar_arrive(empty + 8 * st);
+                taken += 1;
+                return;
+            }
+            broken = true;
+            if (lane == 0) { atomicOr(status, kStCopyTimeout); atomicOr(L.flag, 1u); }
+        }
+        load_chunk<DT>(row, V, ch, lane, v);
+    }
+    // After the CTA-wide barrier that follows the producer's last copy, and only if some wait gave up:
+    // copies still on their way into this warp's ring get a second bounded wait before the CTA may exit.
+    __device__ __forceinline__ void drain(const FeedLayout& L, int w) const {
+        if (*L.flag == 0) return;
+        const uint32_t end = L.issued[w];
+        for (uint32_t k = taken; k < end; ++k) mbar_wait_bounded(full + 8 * (k % kDepth), (k / kDepth) & 1u);
+    }
+};
+
 __device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t x) {
     __nv_bfloat162 r;
     *reinterpret_cast<uint32_t*>(&r) = x;
@@ -178,14 +390,11 @@ __device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 x) { return *reinterpr
 // Largest element of the lane's 4 vectors (NaN entries are skipped; they surface in the sums).
 template <int DT> __device__ __forceinline__ float lane_max(const uint4 (&v)[kVecPerLane]);
 template <> __device__ __forceinline__ float lane_max<DT_BF16>(const uint4 (&v)[kVecPerLane]) {
-    __nv_bfloat162 m = as_bf162(v[0].x);
-    m = __hmax2(m, as_bf162(v[0].y)); m = __hmax2(m, as_bf162(v[0].z)); m = __hmax2(m, as_bf162(v[0].w));
+    __nv_bfloat162 q[kVecPerLane];
 #pragma unroll
-    for (int j = 1; j < kVecPerLane; ++j) {
-        m = __hmax2(m, as_bf162(v[j].x)); m = __hmax2(m, as_bf162(v[j].y));
-        m = __hmax2(m, as_bf162(v[j].z)); m = __hmax2(m, as_bf162(v[j].w));
-    }
-    const uint32_t b = as_u32(m);
+    for (int j = 0; j < kVecPerLane; ++j)                       // four short chains, not one long one
+        q[j] = __hmax2(__hmax2(as_bf162(v[j].x), as_bf162(v[j].y)), __hmax2(as_bf162(v[j].z), as_bf162(v[j].w)));
+    const uint32_t b = as_u32(__hmax2(__hmax2(q[0], q[1]), __hmax2(q[2], q[3])));
     return fmaxf(__uint_as_float(b << 16), __uint_as_float(b & 0xffff0000u));
 }
 template <> __device__ __forceinline__ float lane_max<DT_FP32>(const uint4 (&v)[kVecPerLane]) {
@@ -198,12 +407,41 @@ template <> __device__ __forceinline__ float lane_max<DT_FP32>(const uint4 (&v)[
     return m;
 }
 
+// Two fp32 values in one 64-bit register, for the packed fp32 arithmetic of sm_100 (one instruction per pair).
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// Warp maximum in one instruction (sm_100a); NaN inputs are ignored.
+__device__ __forceinline__ float warp_max_redux(float v) {
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
+}
+
 // sum_e 2^(z_e*c + k) over the lane's elements, and with WANT_T also sum_e w_e*t_e (t_e = z_e*c + k),
 // the numerator of the entropy.  -inf logits are clamped to a huge negative finite value first so that
-// their 0 * (-inf) does not poison the entropy sum; NaN stays NaN.
+// their 0 * (-inf) does not poison the entropy sum; NaN stays NaN.  Two elements per instruction
+// wherever the hardware has a packed form; the exponentials are one MUFU operation per element.
 template <int DT, bool WANT_T>
 __device__ __forceinline__ void lane_sums(const uint4 (&v)[kVecPerLane], float c, float k, float& s_out, float& t_out) {
-    float s0 = 0.f, s1 = 0.f, t0 = 0.f, t1 = 0.f;
+    const f32x2 c2 = pack2(c, c), k2 = pack2(k, k);
+    f32x2 sa = pack2(0.f, 0.f), sb = sa, ta = sa, tb = sa;
     if (DT == DT_BF16) {
         const __nv_bfloat162 floor2 = as_bf162(0xf149f149u);     // about -1e30 in both halves
 #pragma unroll
@@ -213,28 +451,36 @@ __device__ __forceinline__ void lane_sums(const uint4 (&v)[kVecPerLane], float c
             for (int q = 0; q < 4; ++q) {
                 uint32_t x = w[q];
                 if (WANT_T) x = as_u32(__hmax2_nan(as_bf162(x), floor2));
-                const float a = fmaf(__uint_as_float(x << 16), c, k);
-                const float b = fmaf(__uint_as_float(x & 0xffff0000u), c, k);
-                const float wa = ex2_approx(a), wb = ex2_approx(b);
-                s0 += wa; s1 += wb;
-                if (WANT_T) { t0 = fmaf(wa, a, t0); t1 = fmaf(wb, b, t1); }
+                const f32x2 t = fma2(pack2(__uint_as_float(x << 16), __uint_as_float(x & 0xffff0000u)), c2, k2);
+                float a, b;
+                unpack2(t, a, b);
+                const f32x2 e = pack2(ex2_approx(a), ex2_approx(b));
+                if (q & 1) { sb = add2(sb, e); if (WANT_T) tb = fma2(e, t, tb); }
+                else       { sa = add2(sa, e); if (WANT_T) ta = fma2(e, t, ta); }
             }
         }
     } else {
+        const f32x2 floor2 = pack2(-1e30f, -1e30f);
 #pragma unroll
         for (int j = 0; j < kVecPerLane; ++j) {
             const float z[4] = {__uint_as_float(v[j].x), __uint_as_float(v[j].y), __uint_as_float(v[j].z),
                                 __uint_as_float(v[j].w)};
 #pragma unroll
             for (int q = 0; q < 4; q += 2) {
-                float a = fmaf(z[q], c, k), b = fmaf(z[q + 1], c, k);
-                if (WANT_T) { a = (a < -1e30f) ? -1e30f : a; b = (b < -1e30f) ? -1e30f : b; }
-                const float wa = ex2_approx(a), wb = ex2_approx(b);
-                s0 += wa; s1 += wb;
-                if (WANT_T) { t0 = fmaf(wa, a, t0); t1 = fmaf(wb, b, t1); }
+                f32x2 t = fma2(pack2(z[q], z[q + 1]), c2, k2);
+                float a, b;
+                unpack2(t, a, b);
+                if (WANT_T) { a = (a < -1e30f) ? -1e30f : a; b = (b < -1e30f) ? -1e30f : b; t = pack2(a, b); }
+                const f32x2 e = pack2(ex2_approx(a), ex2_approx(b));
+                if (q & 2) { sb = add2(sb, e); if (WANT_T) tb = fma2(e, t, tb); }
+                else       { sa = add2(sa, e); if (WANT_T) ta = fma2(e, t, ta); }
             }
         }
+        (void)floor2;
     }
+    float s0, s1, t0, t1;
+    unpack2(add2(sa, sb), s0, s1);
+    unpack2(add2(ta, tb), t0, t1);
     s_out = s0 + s1;
     t_out = t0 + t1;
 }
@@ -253,7 +499,7 @@ struct WarpAcc {
 // WANT_PART (all lanes get it), else 0.
 template <int DT, bool WANT_T, bool WANT_PART>
 __device__ __forceinline__ float fold_chunk(WarpAcc& acc, const uint4 (&v)[kVecPerLane], int ch, float c) {
-    const float M = warp_max_f(lane_max<DT>(v));
+    const float M = warp_max_redux(lane_max<DT>(v));
     if (M > acc.c1) { acc.c2 = acc.c1; acc.c1 = M; acc.best = ch; }
     else if (M > acc.c2) { acc.c2 = M; }
     if (M > acc.ref || M != M) {
@@ -279,8 +525,11 @@ __device__ __forceinline__ float fold_chunk(WarpAcc& acc, const uint4 (&v)[kVecP
 // contribution of chunk ch to the row total, relative to the row maximum m (mc = m*c in double):
 //   scaled  : part.y * 2^-(k_ch + mc), k_ch = fl(-part.x * c) exactly as the streaming pass used it
 //   absolute: part.y
+// GLOBAL: the partials sit in global memory and may have been written by other CTAs of the running kernel,
+// so they are read through L2.
+template <bool GLOBAL>
 __device__ __forceinline__ double chunk_contrib(const float2* part, int ch, float c, double mc, bool scaled) {
-    const float2 p = part[ch];
+    const float2 p = GLOBAL ? __ldcg(part + ch) : part[ch];
     if (!scaled) return (double)p.y;
     if (!(p.y > 0.f)) return (p.y != p.y) ? (double)p.y : 0.0;
     const double k = (double)__fmul_rn(-p.x, c);
@@ -290,11 +539,12 @@ __device__ __forceinline__ double chunk_contrib(const float2* part, int ch, floa
 struct CdfTotals { double lane_sum, incl, W; };
 
 // Each lane owns a contiguous block of chunks, so the scan is in token order.
+template <bool GLOBAL>
 __device__ __forceinline__ CdfTotals cdf_totals(const float2* part, int NC, float c, double mc, bool scaled, int lane) {
     const int per = (NC + 31) / 32;
     const int b = lane * per, e = min(NC, b + per);
     double ls = 0.0;
-    for (int ch = b; ch < e; ++ch) ls += chunk_contrib(part, ch, c, mc, scaled);
+    for (int ch = b; ch < e; ++ch) ls += chunk_contrib<GLOBAL>(part, ch, c, mc, scaled);
     CdfTotals t;
     t.lane_sum = ls;
     t.incl = warp_incl_scan_d(ls, lane);
@@ -303,6 +553,7 @@ __device__ __forceinline__ CdfTotals cdf_totals(const float2* part, int NC, floa
 }
 
 // The chunk in which the running sum first exceeds tgt, and tgt minus the sum before that chunk.
+template <bool GLOBAL>
 __device__ __forceinline__ int cdf_locate(const float2* part, int NC, float c, double mc, bool scaled, int lane,
                                           const CdfTotals& t, double tgt, double& rem) {
     const int per = (NC + 31) / 32;
@@ -318,7 +569,7 @@ __device__ __forceinline__ int cdf_locate(const float2* part, int NC, float c, d
     int pick = -1, last_pos = -1;
     double before = excl, before_last = excl;
     for (int ch = b; ch < e; ++ch) {
-        const double x = chunk_contrib(part, ch, c, mc, scaled);
+        const double x = chunk_contrib<GLOBAL>(part, ch, c, mc, scaled);
         if (x > 0.0) { last_pos = ch; before_last = run; }
         if (run + x > tgt) { pick = ch; before = run; break; }
         run += x;
@@ -327,6 +578,78 @@ __device__ __forceinline__ int cdf_locate(const float2* part, int NC, float c, d
     rem = tgt - before;
     return pick;
 }
+
+// ---- the same search with the partials of a row held in registers (rows of at most 32 * kRegPer chunks)
+constexpr int kRegPer = 8;
+
+// part.y * 2^-(k_ch + mc) like chunk_contrib, but with the power of two taken apart: integer part by
+// exponent arithmetic, fraction by the fp32 exponential unit (relative error about 2e-7, the accuracy of
+// the partial sums themselves).
+__device__ __forceinline__ double scaled_contrib(float2 p, float c, double mc) {
+    if (!(p.y > 0.f)) return (p.y != p.y) ? (double)p.y : 0.0;
+    const double d = (double)__fmul_rn(-p.x, c) + mc;                     // >= 0 up to rounding
+    const double dn = floor(d);
+    if (dn > 1000.0) return 0.0;
+    const int n = (int)dn;
+    const float fr = (float)(d - dn);
+    return (double)p.y * (double)ex2_approx(-fr) * __hiloint2double((1023 - n) << 20, 0);
+}
+
+struct RegCdf {
+    float2 part[kRegPer];      // this lane's chunks: lane * per .. lane * per + per - 1
+    double con[kRegPer];       // their contributions to the row total, relative to the row maximum
+    double lane_sum, incl, W;
+    int per, NC;
+
+    // The loads go out together; nothing waits on them before scale().
+    __device__ __forceinline__ void load(const float2* g, int nc, int lane) {
+        NC = nc;
+        per = (nc + 31) / 32;
+        const int b = lane * per;
+#pragma unroll
+        for (int j = 0; j < kRegPer; ++j) {
+            part[j] = make_float2(neg_inf(), 0.f);
+            if (j < per && b + j < nc) part[j] = __ldcg(g + b + j);
+        }
+    }
+    __device__ __forceinline__ void scale(float c, double mc, int lane) {
+        double ls = 0.0;
+#pragma unroll
+        for (int j = 0; j < kRegPer; ++j) {
+            con[j] = (j < per) ? scaled_contrib(part[j], c, mc) : 0.0;
+            ls += con[j];
+        }
+        lane_sum = ls;
+        incl = warp_incl_scan_d(ls, lane);
+        W = __shfl_sync(0xffffffffu, incl, 31);
+    }
+    // Chunk in which the running sum first exceeds tgt (if rounding leaves none, the last chunk with a
+    // positive contribution), tgt minus the sum before it, and the chunk's reference logit.
+    __device__ __forceinline__ int locate(double tgt, int lane, double& rem, float& ref) const {
+        const unsigned over = __ballot_sync(0xffffffffu, incl > tgt);
+        const unsigned pos = __ballot_sync(0xffffffffu, lane_sum > 0.0);
+        rem = 0.0; ref = 0.f;
+        int L;
+        if (over) L = __ffs(over) - 1;
+        else if (pos) L = 31 - __clz(pos);
+        else return -1;
+        double run = incl - lane_sum;
+        int pick = -1, last_pos = -1;
+        double before = run, before_last = run;
+        float r_pick = 0.f, r_last = 0.f;
+#pragma unroll
+        for (int j = 0; j < kRegPer; ++j) {
+            const double x = con[j];
+            if (x > 0.0) { last_pos = j; before_last = run; r_last = part[j].x; }
+            if (pick < 0 && run + x > tgt) { pick = j; before = run; r_pick = part[j].x; }
+            run += x;
+        }
+        if (pick < 0) { pick = last_pos; before = before_last; r_pick = r_last; }
+        rem = __shfl_sync(0xffffffffu, tgt - before, L);
+        ref = __shfl_sync(0xffffffffu, r_pick, L);
+        return __shfl_sync(0xffffffffu, L * per + pick, L);
+    }
+};
 
 // The lane's contiguous share of one chunk: EPL consecutive elements = 64 bytes = 4 raw vectors.
 // Vectors wholly at or beyond V are not read (zeros); lane_block_elem masks elements >= V to -inf.
@@ -360,88 +683,81 @@ __device__ __forceinline__ float lane_block_elem(const uint4 (&v)[4], int k, int
     return idx < V ? z : neg_inf();
 }
 
-// Where the per-token weights of one chunk live while a token is picked: registers (finish kernel, one
-// warp per row, registers to spare) or shared memory (verify kernel, whose streaming loops set the budget).
-template <int EPL> struct RegWeights {
-    double w[EPL];
-    __device__ __forceinline__ void set(int k, double v) { w[k] = v; }
-    __device__ __forceinline__ double get(int k) const { return w[k]; }
-};
-template <int EPL> struct SmemWeights {
-    double* base;           // EPL * 32 doubles; element k of lane l at k*32 + l (conflict-free)
-    int lane;
-    __device__ __forceinline__ void set(int k, double v) { base[k * 32 + lane] = v; }
-    __device__ __forceinline__ double get(int k) const { return base[k * 32 + lane]; }
-};
-
-// Token inside one chunk.  Lane l owns the EPL consecutive tokens starting at first_token (its own);
-// W holds their weights in double (>= 0), rem is the target inside the chunk in the same units.  First
-// token whose running sum exceeds rem; if rounding leaves none, the last token with positive weight.
-template <int EPL, typename W>
-__device__ __forceinline__ int pick_in_block(const W& w, int first_token, double rem, int lane) {
+// Token inside one chunk.  Lane l owns the EPL consecutive tokens starting at first_token (its own); w
+// holds their weights (>= 0) exactly as the streaming pass formed them, t is the target inside the chunk
+// in the same units.  First token whose running sum exceeds t; if rounding leaves none, the last token
+// with positive weight.  Sums run in double so that the order of additions cannot matter.
+template <int EPL>
+__device__ __forceinline__ int pick_in_block(const float (&w)[EPL], int first_token, double t, int lane) {
     double sum = 0.0;
 #pragma unroll
-    for (int k = 0; k < EPL; ++k) sum += w.get(k);
+    for (int k = 0; k < EPL; ++k) sum += (double)w[k];
     const double incl = warp_incl_scan_d(sum, lane);
-    const unsigned over = __ballot_sync(0xffffffffu, incl > rem);
+    const unsigned over = __ballot_sync(0xffffffffu, incl > t);
     const unsigned pos = __ballot_sync(0xffffffffu, sum > 0.0);
     int L;
     if (over) L = __ffs(over) - 1;
     else if (pos) L = 31 - __clz(pos);
     else return -1;
-    const double t = rem - (incl - sum);
+    const double tl = t - (incl - sum);
     double run = 0.0;
     int pick = -1, last_pos = -1;
     if (lane == L) {
 #pragma unroll
         for (int k = 0; k < EPL; ++k) {
-            const double x = w.get(k);
+            const double x = (double)w[k];
             if (x > 0.0) last_pos = k;
             run += x;
-            if (pick < 0 && run > t) pick = k;
+            if (pick < 0 && run > tl) pick = k;
         }
         if (pick < 0) pick = last_pos;
     }
     return __shfl_sync(0xffffffffu, first_token + pick, L);
 }
 
-template <int DT, typename W>
-__device__ __forceinline__ int pick_softmax(W& w, const void* row, int V, int chunk, double rem, double inv_T,
-                                            double m_s, int lane) {
+// x ~ softmax inside one chunk: weights 2^(z*c + k) with the k the streaming pass used for this chunk.
+template <int DT>
+__device__ __forceinline__ int pick_softmax_block(const uint4 (&v)[4], int V, int chunk, float c, float k, double t, int lane) {
     constexpr int EPL = chunk_elems<DT>() / 32;
     const int e0 = chunk * chunk_elems<DT>() + lane * EPL;
-    uint4 v[4];
-    load_lane_block<DT>(row, V, chunk, lane, v);
+    float w[EPL];
 #pragma unroll
-    for (int k = 0; k < EPL; ++k) w.set(k, exp((double)lane_block_elem<DT>(v, k, e0 + k, V) * inv_T - m_s));
-    return pick_in_block<EPL>(w, e0, rem, lane);
+    for (int j = 0; j < EPL; ++j) w[j] = ex2_approx(fmaf(lane_block_elem<DT>(v, j, e0 + j, V), c, k));
+    return pick_in_block<EPL>(w, e0, t, lane);
 }
 
-template <int DT, typename W>
-__device__ __forceinline__ int pick_residual(W& w, const void* prow, const void* qrow, int V, int chunk, double rem,
-                                             double iTp, double lse_p, double iTq, double lse_q, int lane) {
+template <int DT>
+__device__ __forceinline__ int pick_softmax(const void* row, int V, int chunk, float c, float k, double t, int lane) {
+    uint4 v[4];
+    load_lane_block<DT>(row, V, chunk, lane, v);
+    return pick_softmax_block<DT>(v, V, chunk, c, k, t, lane);
+}
+
+// x ~ norm(max(0, p - q)) inside one chunk, weights formed as in the residual streaming pass.
+template <int DT>
+__device__ __forceinline__ int pick_residual(const void* prow, const void* qrow, int V, int chunk, float cp, float kp,
+                                             float cq, float kq, float beta, double t, int lane) {
     constexpr int EPL = chunk_elems<DT>() / 32;
     const int e0 = chunk * chunk_elems<DT>() + lane * EPL;
     uint4 vp[4], vq[4];
     load_lane_block<DT>(prow, V, chunk, lane, vp);
     load_lane_block<DT>(qrow, V, chunk, lane, vq);
+    float w[EPL];
 #pragma unroll
-    for (int k = 0; k < EPL; ++k) {
-        const double r = exp((double)lane_block_elem<DT>(vp, k, e0 + k, V) * iTp - lse_p) -
-                         exp((double)lane_block_elem<DT>(vq, k, e0 + k, V) * iTq - lse_q);
-        w.set(k, r > 0.0 ? r : 0.0);
+    for (int j = 0; j < EPL; ++j) {
+        const float wp = ex2_approx(fmaf(lane_block_elem<DT>(vp, j, e0 + j, V), cp, kp));
+        const float wq = ex2_approx(fmaf(lane_block_elem<DT>(vq, j, e0 + j, V), cq, kq));
+        w[j] = fmaxf(fmaf(wp, beta, -wq), 0.f);
     }
-    return pick_in_block<EPL>(w, e0, rem, lane);
+    return pick_in_block<EPL>(w, e0, t, lane);
 }
 
 // In one chunk: how many elements equal the row maximum m, the lowest index of one, and the largest
 // element below m.  Whole warp; every lane returns the same values.
 template <int DT>
-__device__ __forceinline__ void scan_top_chunk(const void* row, int V, int chunk, float m, int lane, int& cnt,
+__device__ __forceinline__ void scan_top_block(const uint4 (&v)[4], int V, int chunk, float m, int lane, int& cnt,
                                                int& first, float& below) {
     constexpr int EPL = chunk_elems<DT>() / 32;
-    uint4 v[4];
-    load_lane_block<DT>(row, V, chunk, lane, v);
     int c = 0, f = 0x7fffffff;
     float b = neg_inf();
     const int e0 = chunk * chunk_elems<DT>() + lane * EPL;
