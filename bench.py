@@ -173,6 +173,8 @@ def bench_ours(args):
     dev = tp.Tapout.from_workload(w, seq_offset=rank * S, token_out_stride=K)
     if args.row_segments:
         dev.set_param("row_segments", args.row_segments)
+    if args.verify_cluster:
+        dev.set_param("verify_cluster", args.verify_cluster)
     pool = [si.round_logits(si.scaled(w, seed=w.seed + 1000 * rank), r, device) for r in range(POOL_ROUNDS)]
     toks = torch.full((S, K), -1, dtype=torch.int32, device=device)
     cont = torch.empty(S, dtype=torch.uint8, device=device)
@@ -353,6 +355,7 @@ def main():
     ap.add_argument("--ref-sample-seqs", type=int, default=32)
     ap.add_argument("--n-seq", type=int, default=0, help="override the batch size (profiling captures)")
     ap.add_argument("--row-segments", type=int, default=0, help="CTAs per draft row (0 = library default)")
+    ap.add_argument("--verify-cluster", type=int, default=0, help="CTAs per verify cluster (0 = library default)")
     ap.add_argument("--pool-rounds", type=int, default=POOL_ROUNDS)
     args = ap.parse_args()
     if args.impl == "reference":

@@ -88,10 +88,12 @@ bool stride_ok(const tapout* h, int64_t stride_elems) { return stride_elems > 0 
 
 float c_of(float inv_T) { return (float)((double)inv_T * kLog2e); }
 
-// Largest power-of-two cluster (at most 8 CTAs, the portable limit) that still leaves every warp of a CTA
-// a chunk of its own per row.
-int auto_cluster(int NC) {
-    int cs = kMaxCluster;
+// CTAs per verify cluster when the caller does not say: enough clusters to occupy the device when the
+// batch is small, never fewer than two CTAs per sequence (a single CTA walks a long draft too slowly),
+// never so many that a warp is left without a chunk of its own per row; a power of two, at most 8.
+int auto_cluster(int NC, int n_seq, int resident_ctas) {
+    int cs = 2;
+    while (cs < kMaxCluster && (long long)cs * n_seq < resident_ctas) cs <<= 1;
     while (cs > 1 && NC / cs < kWarps) cs >>= 1;
     return cs;
 }
@@ -121,7 +123,7 @@ int setup_scratch(tapout* h) {
     if (p.nseg > p.NC) p.nseg = p.NC;
 
     // verify clusters: the requested size, reduced until the device can co-schedule such a cluster
-    int cs = h->cluster_user > 0 ? h->cluster_user : auto_cluster(p.NC);
+    int cs = h->cluster_user > 0 ? h->cluster_user : auto_cluster(p.NC, p.S, h->n_sm * kResident);
     if (cs > p.NC) cs = 1;
     for (;; cs >>= 1) {
         h->walk_smem = sizeof(float2) * (size_t)((p.NC + cs - 1) / cs + 1);
@@ -131,10 +133,6 @@ int setup_scratch(tapout* h) {
         if (fit > 0 || cs == 1) break;
     }
     h->cluster = cs;
-    TP_CUDA(h, cudaFuncSetAttribute(k_draft_step<DT_BF16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFeedSmem));
-    TP_CUDA(h, cudaFuncSetAttribute(k_draft_step<DT_FP32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFeedSmem));
-    TP_CUDA(h, cudaFuncSetAttribute(k_draft_step<DT_BF16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFeedSmem));
-    TP_CUDA(h, cudaFuncSetAttribute(k_draft_step<DT_FP32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFeedSmem));
     if (h->walk_smem > 40 * 1024) {
         TP_CUDA(h, cudaFuncSetAttribute(k_verify_walk<DT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
         TP_CUDA(h, cudaFuncSetAttribute(k_verify_walk<DT_FP32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
@@ -161,7 +159,7 @@ int setup_scratch(tapout* h) {
     h->sc.done = reinterpret_cast<int32_t*>(h->d_scratch + o_done);
     h->sc.status = reinterpret_cast<unsigned long long*>(h->d_scratch + o_status);
 
-    h->grid_rows = h->n_sm * 3;                               // persistent: every CTA resident
+    h->grid_rows = h->n_sm * kResident;                       // persistent: every CTA resident
     h->arms_ready = false;
     return TAPOUT_OK;
 }
@@ -222,8 +220,8 @@ int draft_step_impl(tapout* h, const void* logits, int64_t stride, int32_t* out_
     a.out_token = out_token; a.tok_stride = tok_stride; a.out_continue = out_continue;
     const int pk = h->pos == 0 ? 0 : 2;
     { int rc = profile_mark(h, pk); if (rc) return rc; }
-    if (h->p.dtype == DT_BF16) k_draft_step<DT_BF16, false><<<h->grid_rows, kStepThreads, kFeedSmem, h->stream>>>(h->p, h->st, h->sc, a);
-    else k_draft_step<DT_FP32, false><<<h->grid_rows, kStepThreads, kFeedSmem, h->stream>>>(h->p, h->st, h->sc, a);
+    if (h->p.dtype == DT_BF16) k_draft_step<DT_BF16, false><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->st, h->sc, a);
+    else k_draft_step<DT_FP32, false><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->st, h->sc, a);
     TP_LAUNCHED(h);
     { int rc = profile_mark(h, pk); if (rc) return rc; }
     h->pos += 1;
@@ -574,8 +572,8 @@ int tapout_row_stats(tapout_t* h, const void* logits, int n_rows, int64_t row_st
     if (!aligned16(logits) || !stride_ok(h, row_stride) || row_stride < h->p.V) return TAPOUT_E_ALIGNMENT;
     StepArgs a = step_args(h, logits, row_stride, c_of((float)inv_temp));
     a.n_fixed = n_rows; a.inv_T = (float)inv_temp; a.out_feat = out_features;
-    if (h->p.dtype == DT_BF16) k_draft_step<DT_BF16, true><<<h->grid_rows, kStepThreads, kFeedSmem, h->stream>>>(h->p, h->st, h->sc, a);
-    else k_draft_step<DT_FP32, true><<<h->grid_rows, kStepThreads, kFeedSmem, h->stream>>>(h->p, h->st, h->sc, a);
+    if (h->p.dtype == DT_BF16) k_draft_step<DT_BF16, true><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->st, h->sc, a);
+    else k_draft_step<DT_FP32, true><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->st, h->sc, a);
     TP_LAUNCHED(h);
     return TAPOUT_OK;
 }

@@ -170,216 +170,6 @@ __device__ __forceinline__ void load_chunk(const void* row, int V, int ch, int l
     }
 }
 
-// ------------------------------------------------------------------ asynchronous chunk pipeline
-// Each warp keeps kDepth full 2 KB chunks on their way from global to its own ring in shared memory:
-// one lane issues a bulk asynchronous copy per chunk (the TMA unit moves the bytes, no registers are
-// held), completion is signalled on an mbarrier of the warp's own.  A chunk that reaches past the end of
-// the row is not copied this way: it is read with plain loads.  Every wait is bounded; if one gives up
-// the warp records it in the status word and reads this and all later chunks with plain loads.
-constexpr int kDepth = 4;
-constexpr int kChunkBytes = 32 * kVecPerLane * 16;
-constexpr int kRingBytes = kWarps * kDepth * kChunkBytes;       // per CTA
-constexpr int kPipeSmem = kRingBytes + kWarps * kDepth * 8;     // ring + mbarriers
-constexpr int kWaitTries = 1 << 22;
-constexpr unsigned long long kStCopyTimeout = 16ull;
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
-
-template <int DT> __device__ __forceinline__ bool chunk_is_full(int V, int ch) { return (ch + 1) * chunk_elems<DT>() <= V; }
-
-struct WarpPipe {
-    uint32_t data, bars;          // shared-space addresses of this warp's ring and of its kDepth mbarriers
-    uint32_t issued, taken;       // full chunks issued / taken so far
-    bool broken;
-
-    // ring: kRingBytes, 128-byte aligned; bar: kWarps * kDepth words of 8 bytes.  Call once per kernel, all lanes.
-    __device__ __forceinline__ void init(unsigned char* ring, unsigned long long* bar, int warp, int lane) {
-        data = smem_u32(ring) + (uint32_t)warp * kDepth * kChunkBytes;
-        bars = smem_u32(bar) + (uint32_t)warp * kDepth * 8;
-        issued = taken = 0;
-        broken = false;
-        if (lane == 0) {
-#pragma unroll
-            for (int d = 0; d < kDepth; ++d) mbar_init(bars + 8 * d, 1);
-            fence_proxy_async();
-        }
-        __syncwarp();
-    }
-    __device__ __forceinline__ int in_flight() const { return (int)(issued - taken); }
-    // src: 16-byte aligned start of a full chunk.  Needs in_flight() < kDepth.
-    __device__ __forceinline__ void issue(const void* src, int lane) {
-        if (broken) return;
-        __syncwarp();                                  // every lane has read the stage that is overwritten now
-        const uint32_t st = issued % kDepth;
-        if (lane == 0) {
-            fence_proxy_async();
-            mbar_expect_tx(bars + 8 * st, kChunkBytes);
-            bulk_g2s(data + st * kChunkBytes, src, kChunkBytes, bars + 8 * st);
-        }
-        issued += 1;
-    }
-    __device__ __forceinline__ bool wait_stage(uint32_t k) const {
-        const uint32_t bar = bars + 8 * (k % kDepth), parity = (k / kDepth) & 1u;
-        bool ok = false;
-        for (int it = 0; it < kWaitTries && !ok; ++it) ok = mbar_try_wait(bar, parity);
-        return __all_sync(0xffffffffu, ok);
-    }
-    // The oldest chunk in flight, in the lane layout of load_chunk.  row / ch name the same chunk for the
-    // fallback path.
-    template <int DT>
-    __device__ __forceinline__ void take(const void* row, int V, int ch, int lane, uint4 (&v)[kVecPerLane],
-                                         unsigned long long* status) {
-        if (!broken) {
-            if (wait_stage(taken)) {
-                const uint32_t base = data + (taken % kDepth) * kChunkBytes + (uint32_t)lane * 16;
-#pragma unroll
-                for (int j = 0; j < kVecPerLane; ++j) v[j] = lds128(base + j * 512);
-                taken += 1;
-                return;
-            }
-            broken = true;
-            if (lane == 0) atomicOr(status, kStCopyTimeout);
-        }
-        load_chunk<DT>(row, V, ch, lane, v);
-    }
-    // Before the CTA exits after a wait gave up: its copies still in flight are given a second bounded wait.
-    __device__ __forceinline__ void drain() const {
-        if (!broken) return;
-        for (uint32_t k = taken; k != issued; ++k) wait_stage(k);
-    }
-};
-
-// ---- the same ring fed by a producer: one extra warp per CTA issues the copies (lane w feeds the ring
-// of folding warp w and runs ahead of it by up to kDepth chunks, across work items), the folding warps
-// only wait, read and hand the stage back.  full[w][d]: copy landed (1 arrival + 2048 bytes);
-// empty[w][d]: all 32 lanes of warp w have read the stage.
-constexpr int kFeedSmem = kRingBytes + 2 * kWarps * kDepth * 8 + 64;     // ring, full, empty, issued counts, flag
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-struct FeedLayout {
-    unsigned char* ring;
-    unsigned long long* full;
-    unsigned long long* empty;
-    uint32_t* issued;            // [kWarps] chunks each producer lane has issued, written when it is done
-    uint32_t* flag;              // nonzero once any wait gave up
-    __device__ __forceinline__ explicit FeedLayout(unsigned char* base) {
-        ring = base;
-        full = reinterpret_cast<unsigned long long*>(base + kRingBytes);
-        empty = full + kWarps * kDepth;
-        issued = reinterpret_cast<uint32_t*>(empty + kWarps * kDepth);
-        flag = issued + kWarps;
-    }
-    // All threads of the CTA; followed by a CTA-wide barrier at the caller.
-    __device__ __forceinline__ void init(int tid) const {
-        if (tid < kWarps * kDepth) {
-            mbar_init(smem_u32(full + tid), 1);
-            mbar_init(smem_u32(empty + tid), 32);
-        }
-        if (tid < kWarps) issued[tid] = 0;
-        if (tid == 0) *flag = 0;
-        fence_proxy_async();
-    }
-};
-
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    bool ok = false;
-    for (int it = 0; it < kWaitTries && !ok; ++it) ok = mbar_try_wait(bar, parity);
-    return ok;
-}
-
-// One lane of the producer warp.
-struct FeedProducer {
-    uint32_t data, full, empty, n;
-    bool dead;
-    __device__ __forceinline__ void init(const FeedLayout& L, int w) {
-        data = smem_u32(L.ring) + (uint32_t)w * kDepth * kChunkBytes;
-        full = smem_u32(L.full + w * kDepth);
-        empty = smem_u32(L.empty + w * kDepth);
-        n = 0;
-        dead = false;
-    }
-    // src: 16-byte aligned start of a full chunk.  Waits until the stage it goes to has been read.
-    __device__ __forceinline__ void issue(const void* src, const FeedLayout& L, unsigned long long* status) {
-        if (dead) return;
-        const uint32_t st = n % kDepth;
-        if (n >= kDepth && !mbar_wait_bounded(empty + 8 * st, ((n / kDepth) - 1u) & 1u)) {
-            dead = true;
-            atomicOr(status, kStCopyTimeout);
-            atomicOr(L.flag, 1u);
-            return;
-        }
-        mbar_expect_tx(full + 8 * st, kChunkBytes);
-        bulk_g2s(data + st * kChunkBytes, src, kChunkBytes, full + 8 * st);
-        n += 1;
-    }
-};
-
-// A folding warp (all 32 lanes).
-struct FeedConsumer {
-    uint32_t data, full, empty, taken;
-    bool broken;
-    __device__ __forceinline__ void init(const FeedLayout& L, int w) {
-        data = smem_u32(L.ring) + (uint32_t)w * kDepth * kChunkBytes;
-        full = smem_u32(L.full + w * kDepth);
-        empty = smem_u32(L.empty + w * kDepth);
-        taken = 0;
-        broken = false;
-    }
-    // The warp's next full chunk, in the lane layout of load_chunk.  row / ch name the same chunk for the
-    // plain-load path that takes over once a wait has given up.
-    template <int DT>
-    __device__ __forceinline__ void take(const void* row, int V, int ch, int lane, uint4 (&v)[kVecPerLane],
-                                         const FeedLayout& L, unsigned long long* status) {
-        if (!broken) {
-            const uint32_t st = taken % kDepth;
-            const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(full + 8 * st, (taken / kDepth) & 1u));
-            if (ok) {
-                const uint32_t base = data + st * kChunkBytes + (uint32_t)lane * 16;
-#pragma unroll
-                for (int j = 0; j < kVecPerLane; ++j) v[j] = lds128(base + j * 512);
-                mbar_arrive(empty + 8 * st);
-                taken += 1;
-                return;
-            }
-            broken = true;
-            if (lane == 0) { atomicOr(status, kStCopyTimeout); atomicOr(L.flag, 1u); }
-        }
-        load_chunk<DT>(row, V, ch, lane, v);
-    }
-    // After the CTA-wide barrier that follows the producer's last copy, and only if some wait gave up:
-    // copies still on their way into this warp's ring get a second bounded wait before the CTA may exit.
-    __device__ __forceinline__ void drain(const FeedLayout& L, int w) const {
-        if (*L.flag == 0) return;
-        const uint32_t end = L.issued[w];
-        for (uint32_t k = taken; k < end; ++k) mbar_wait_bounded(full + 8 * (k % kDepth), (k / kDepth) & 1u);
-    }
-};
-
 __device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t x) {
     __nv_bfloat162 r;
     *reinterpret_cast<uint32_t*>(&r) = x;
@@ -434,6 +224,18 @@ __device__ __forceinline__ float warp_max_redux(float v) {
     return r;
 }
 
+// The two bf16 halves of a word as fp32, one byte-permute each.
+__device__ __forceinline__ float bf16_lo(uint32_t x) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, 0, 0x1044;" : "=r"(r) : "r"(x));
+    return __uint_as_float(r);
+}
+__device__ __forceinline__ float bf16_hi(uint32_t x) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, 0, 0x3244;" : "=r"(r) : "r"(x));
+    return __uint_as_float(r);
+}
+
 // sum_e 2^(z_e*c + k) over the lane's elements, and with WANT_T also sum_e w_e*t_e (t_e = z_e*c + k),
 // the numerator of the entropy.  -inf logits are clamped to a huge negative finite value first so that
 // their 0 * (-inf) does not poison the entropy sum; NaN stays NaN.  Two elements per instruction
@@ -451,7 +253,7 @@ __device__ __forceinline__ void lane_sums(const uint4 (&v)[kVecPerLane], float c
             for (int q = 0; q < 4; ++q) {
                 uint32_t x = w[q];
                 if (WANT_T) x = as_u32(__hmax2_nan(as_bf162(x), floor2));
-                const f32x2 t = fma2(pack2(__uint_as_float(x << 16), __uint_as_float(x & 0xffff0000u)), c2, k2);
+                const f32x2 t = fma2(pack2(bf16_lo(x), bf16_hi(x)), c2, k2);
                 float a, b;
                 unpack2(t, a, b);
                 const f32x2 e = pack2(ex2_approx(a), ex2_approx(b));
@@ -500,9 +302,8 @@ struct WarpAcc {
 template <int DT, bool WANT_T, bool WANT_PART>
 __device__ __forceinline__ float fold_chunk(WarpAcc& acc, const uint4 (&v)[kVecPerLane], int ch, float c) {
     const float M = warp_max_redux(lane_max<DT>(v));
-    if (M > acc.c1) { acc.c2 = acc.c1; acc.c1 = M; acc.best = ch; }
-    else if (M > acc.c2) { acc.c2 = M; }
-    if (M > acc.ref || M != M) {
+    if (M > acc.ref) {
+        // a new running maximum (rare after the first chunks): the sums move to the new reference
         const float kn = __fmul_rn(-M, c);
         if (acc.ref > neg_inf()) {
             const float dd = kn - acc.k;                  // <= 0, exact
@@ -510,10 +311,13 @@ __device__ __forceinline__ float fold_chunk(WarpAcc& acc, const uint4 (&v)[kVecP
             if (WANT_T) acc.T = f * fmaf(dd, acc.S, acc.T);
             acc.S *= f;
         }
-        acc.ref = M;
+        acc.c2 = acc.ref;
+        acc.ref = M; acc.c1 = M; acc.best = ch;
         acc.k = kn;
+    } else {
+        acc.c2 = fmaxf(acc.c2, M);
     }
-    if (acc.ref == neg_inf()) return 0.f;                  // nothing finite yet (a NaN reference falls through on purpose)
+    // While nothing finite has been seen k is still 0 and every term below is exactly 0.
     float sc, tc;
     lane_sums<DT, WANT_T>(v, c, acc.k, sc, tc);
     acc.S += sc;

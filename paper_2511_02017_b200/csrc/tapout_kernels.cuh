@@ -19,7 +19,7 @@ namespace tpo {
 namespace cg = cooperative_groups;
 
 constexpr int kMaxCluster = 8;           // portable cluster size limit
-constexpr int kStepThreads = kThreads + 32;  // draft step CTA: the folding warps and one producer warp
+constexpr int kResident = 4;              // CTAs of a streaming kernel resident per SM (64 registers per thread)
 constexpr int kTodo = 32;                // rows a CTA may queue for finishing after its streaming loop
 
 struct WarpRec { float ref, k, S, T, c1, c2; int best; int pad; };
@@ -29,36 +29,33 @@ struct WarpRec { float ref, k, S, T, c1, c2; int best; int pad; };
 // number of waves of the persistent grid, else the best-filling one; never less than a chunk per warp.
 __device__ __forceinline__ int segments_for(const Params& p, int n_rows, int grid) {
     if (p.nseg > 0) return p.nseg;
-    const int cap = max(1, min(min(kMaxSeg, p.NC), max(p.NC / kWarps, 1)));
+    const unsigned cap = (unsigned)max(1, min(min(kMaxSeg, p.NC), max(p.NC / kWarps, 1)));
     if (n_rows <= 0) return 1;
-    int best = 1;
-    long long best_num = 0, best_den = 1;                // fill of `best` = best_num / best_den
-    for (int k = 1; k <= cap; ++k) {
-        const long long items = (long long)n_rows * k;
-        const long long slots = (items + grid - 1) / grid * grid;
-        if (items * 10 >= slots * 9) return k;
-        if (items * best_den > best_num * slots) { best = k; best_num = items; best_den = slots; }
+    const unsigned n = (unsigned)n_rows, G = (unsigned)grid;     // n * cap < 2^31: n_seq is bounded at create
+    unsigned best = 1;
+    float best_fill = 0.f;
+    for (unsigned k = 1; k <= cap; ++k) {
+        const unsigned items = n * k;
+        const unsigned slots = (items + G - 1) / G * G;
+        const float fill = (float)items / (float)slots;
+        if (fill >= 0.9f) return (int)k;
+        if (fill > best_fill) { best = k; best_fill = fill; }
     }
-    return best;
+    return (int)best;
 }
 
-// One warp's share of the chunks [c0, c1) of a row: chunk c0 + warp, then every kWarps-th.  The loads of
-// the next chunk are in flight while the current one is folded.  store(ch, ref, total) receives the
-// per-chunk partial sum when WANT_PART.
+// One warp's share of the chunks [c0, c1) of a row: chunk c0 + warp, then every kWarps-th.  Loads are not
+// staged ahead: with four CTAs resident per SM the other warps cover the latency, and the registers a
+// second buffer would take cost more than it gains.  store(ch, ref, total) receives the per-chunk partial
+// sum when WANT_PART.
 template <int DT, bool WANT_T, bool WANT_PART, typename Store>
 __device__ __forceinline__ void stream_chunks(WarpAcc& acc, const void* row, int V, int c0, int c1, int warp, int lane,
                                               float c, Store store) {
-    int ch = c0 + warp;
-    uint4 cur[kVecPerLane], nxt[kVecPerLane];
-    if (ch < c1) load_chunk<DT>(row, V, ch, lane, cur);
-    while (ch < c1) {
-        const int chn = ch + kWarps;
-        if (chn < c1) load_chunk<DT>(row, V, chn, lane, nxt);
-        const float tot = fold_chunk<DT, WANT_T, WANT_PART>(acc, cur, ch, c);
+    for (int ch = c0 + warp; ch < c1; ch += kWarps) {
+        uint4 v[kVecPerLane];
+        load_chunk<DT>(row, V, ch, lane, v);
+        const float tot = fold_chunk<DT, WANT_T, WANT_PART>(acc, v, ch, c);
         if (WANT_PART && lane == 0) store(ch, acc.ref, tot);
-#pragma unroll
-        for (int j = 0; j < kVecPerLane; ++j) cur[j] = nxt[j];
-        ch = chn;
     }
 }
 
@@ -224,17 +221,14 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
 // another one.  FEATURES: rows 0 .. n_fixed-1 instead of the drafting list, features to out_feat.
 // ============================================================================================
 template <int DT, bool FEATURES>
-__global__ void __launch_bounds__(kStepThreads, 3)
+__global__ void __launch_bounds__(kThreads, kResident)
 k_draft_step(Params p, State st, Scratch sc, StepArgs a)
 {
     constexpr int ESZ = Elem<DT>::BYTES;
-    extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ WarpRec wrec[2][kWarps];
     __shared__ int todo[kTodo];              // rows whose last segment this CTA reduced: finished after the streaming
     __shared__ int n_todo;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const FeedLayout feed(dyn_smem);
-    feed.init(tid);
     if (tid == 0) n_todo = 0;
     const int n_rows = FEATURES ? a.n_fixed : sc.count[a.slot];
     const int32_t* list = sc.list + (size_t)a.slot * p.S;
@@ -242,111 +236,74 @@ k_draft_step(Params p, State st, Scratch sc, StepArgs a)
         // the list two positions ahead is free again: nobody reads or appends to it during this launch
         if (blockIdx.x == 0 && tid == 0) sc.count[(a.slot + 2) % 3] = 0;
         // sequences that stopped at an earlier position draft nothing
-        for (int s = blockIdx.x * kStepThreads + tid; s < p.S; s += gridDim.x * kStepThreads)
+        for (int s = blockIdx.x * kThreads + tid; s < p.S; s += gridDim.x * kThreads)
             if (sc.next_pos[s] < a.pos) { a.out_token[(size_t)s * a.tok_stride] = -1; a.out_continue[s] = 0; }
     }
     const int nseg = segments_for(p, n_rows, (int)gridDim.x);
     const int total = n_rows * nseg;
     const float c = a.c;
-    __syncthreads();
 
-    auto item_row = [&](int item, int& s, int& g) -> const char* {
-        const int ai = item / nseg;
-        g = item - ai * nseg;
-        s = FEATURES ? ai : list[ai];
-        return reinterpret_cast<const char*>(a.logits) + (size_t)s * a.row_stride * ESZ;
-    };
-    auto seg_lo = [&](int g) { return (int)(((long long)g * p.NC) / nseg); };
+    int it = 0;
+    for (int item = blockIdx.x; item < total; item += gridDim.x, ++it) {
+        const int ai = item / nseg, g = item - ai * nseg;
+        const int s = FEATURES ? ai : list[ai];
+        const char* row = reinterpret_cast<const char*>(a.logits) + (size_t)s * a.row_stride * ESZ;
+        const int c0 = (int)(((long long)g * p.NC) / nseg);
+        const int c1 = (int)(((long long)(g + 1) * p.NC) / nseg);
+        float2* part = sc.cdf + (size_t)s * p.NC;
 
-    if (warp == kWarps) {
-        // ---- producer warp: lane w walks folding warp w's chunks in order and keeps its ring full
-        if (lane < kWarps) {
-            FeedProducer prod;
-            prod.init(feed, lane);
-            for (int item = blockIdx.x; item < total && !prod.dead; item += gridDim.x) {
-                int s, g;
-                const char* row = item_row(item, s, g);
-                const int c1 = seg_lo(g + 1);
-                for (int ch = seg_lo(g) + lane; ch < c1; ch += kWarps)
-                    if (chunk_is_full<DT>(p.V, ch)) prod.issue(row + (size_t)ch * kChunkBytes, feed, &sc.status[0]);
-            }
-            feed.issued[lane] = prod.n;
+        WarpAcc acc;
+        acc.init();
+        stream_chunks<DT, true, true>(acc, row, p.V, c0, c1, warp, lane, c,
+                                      [&](int ch, float ref, float tot) { part[ch] = make_float2(ref, tot); });
+        const float Sw = warp_sum_f(acc.S), Tw = warp_sum_f(acc.T);
+        const int buf = it & 1;
+        if (lane == 0) {
+            WarpRec r;
+            r.ref = acc.ref; r.k = acc.k; r.S = Sw; r.T = Tw; r.c1 = acc.c1; r.c2 = acc.c2; r.best = acc.best; r.pad = 0;
+            wrec[buf][warp] = r;
         }
-    } else {
-        // ---- folding warps
-        FeedConsumer cons;
-        cons.init(feed, warp);
-        int it = 0;
-        for (int item = blockIdx.x; item < total; item += gridDim.x, ++it) {
-            int s, g;
-            const char* row = item_row(item, s, g);
-            const int c1 = seg_lo(g + 1);
-            float2* part = sc.cdf + (size_t)s * p.NC;
-
-            WarpAcc acc;
-            acc.init();
-            for (int ch = seg_lo(g) + warp; ch < c1; ch += kWarps) {
-                uint4 v[kVecPerLane];
-                if (chunk_is_full<DT>(p.V, ch)) cons.take<DT>(row, p.V, ch, lane, v, feed, &sc.status[0]);
-                else load_chunk<DT>(row, p.V, ch, lane, v);
-                const float tot = fold_chunk<DT, true, true>(acc, v, ch, c);
-                if (lane == 0) part[ch] = make_float2(acc.ref, tot);
-            }
-            const float Sw = warp_sum_f(acc.S), Tw = warp_sum_f(acc.T);
-            const int buf = it & 1;
+        __syncthreads();                     // also orders every warp's chunk partials before the fence below
+        if (warp == (it & (kWarps - 1))) {   // the merging warp rotates; the others run ahead into the next item
+            // lane w merges warp w's record: common reference = the largest, sums rescaled to it
+            WarpRec r;
+            r.ref = neg_inf(); r.k = 0.f; r.S = 0.f; r.T = 0.f; r.c1 = neg_inf(); r.c2 = neg_inf(); r.best = -1;
+            if (lane < kWarps) r = wrec[buf][lane];
+            const bool live = r.ref != neg_inf();                 // a NaN reference counts as live and poisons S
+            const float ref = warp_max_f(r.ref);
+            const float kref = __fmul_rn(-ref, c);
+            const float dd = live ? kref - r.k : 0.f;             // <= 0
+            const float f = live ? ex2_approx(dd) : 0.f;
+            const float Sg = warp_sum_f(live ? f * r.S : 0.f);
+            const float Tg = warp_sum_f(live ? f * fmaf(dd, r.S, r.T) : 0.f);
+            // two largest chunk maxima of the segment (with multiplicity); lowest chunk holding the largest
+            const unsigned tie = __ballot_sync(0xffffffffu, r.best >= 0 && r.c1 == ref);
+            const int win = tie ? __ffs(tie) - 1 : 0;
+            const float other = warp_max_f((lane == win) ? neg_inf() : r.c1);
+            const float c2all = warp_max_f(r.c2);
+            const float C2 = (__popc(tie) >= 2) ? ref : fmaxf(other, c2all);
+            const int best = __reduce_min_sync(0xffffffffu, (tie >> lane) & 1u ? r.best : 0x7fffffff);
+            int last = 0;
             if (lane == 0) {
-                WarpRec r;
-                r.ref = acc.ref; r.k = acc.k; r.S = Sw; r.T = Tw; r.c1 = acc.c1; r.c2 = acc.c2; r.best = acc.best; r.pad = 0;
-                wrec[buf][warp] = r;
+                SegRec o;
+                o.ref = ref; o.S = Sg; o.T = Tg; o.c2 = C2; o.best = (best == 0x7fffffff) ? -1 : best;
+                o.pad0 = o.pad1 = o.pad2 = 0;
+                store_segrec(sc.seg + (size_t)s * kMaxSeg + g, o);
+                __threadfence();             // the segment (record and chunk partials) before it is counted
+                last = atomicAdd(&sc.done[s], 1) == nseg - 1;
+                if (last && n_todo < kTodo) { todo[n_todo] = s; n_todo = n_todo + 1; last = 0; }
             }
-            // the folding warps only; also orders every warp's chunk partials before the fence below
-            asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
-            if (warp == (it & (kWarps - 1))) {   // the merging warp rotates; the others run ahead into the next item
-                // lane w merges warp w's record: common reference = the largest, sums rescaled to it
-                WarpRec r;
-                r.ref = neg_inf(); r.k = 0.f; r.S = 0.f; r.T = 0.f; r.c1 = neg_inf(); r.c2 = neg_inf(); r.best = -1;
-                if (lane < kWarps) r = wrec[buf][lane];
-                const bool live = r.ref != neg_inf();                 // a NaN reference counts as live and poisons S
-                const float ref = warp_max_f(r.ref);
-                const float kref = __fmul_rn(-ref, c);
-                const float dd = live ? kref - r.k : 0.f;             // <= 0
-                const float f = live ? ex2_approx(dd) : 0.f;
-                const float Sg = warp_sum_f(live ? f * r.S : 0.f);
-                const float Tg = warp_sum_f(live ? f * fmaf(dd, r.S, r.T) : 0.f);
-                // two largest chunk maxima of the segment (with multiplicity); lowest chunk holding the largest
-                const unsigned tie = __ballot_sync(0xffffffffu, r.best >= 0 && r.c1 == ref);
-                const int win = tie ? __ffs(tie) - 1 : 0;
-                const float other = warp_max_f((lane == win) ? neg_inf() : r.c1);
-                const float c2all = warp_max_f(r.c2);
-                const float C2 = (__popc(tie) >= 2) ? ref : fmaxf(other, c2all);
-                const int best = __reduce_min_sync(0xffffffffu, (tie >> lane) & 1u ? r.best : 0x7fffffff);
-                int last = 0;
-                if (lane == 0) {
-                    SegRec o;
-                    o.ref = ref; o.S = Sg; o.T = Tg; o.c2 = C2; o.best = (best == 0x7fffffff) ? -1 : best;
-                    o.pad0 = o.pad1 = o.pad2 = 0;
-                    store_segrec(sc.seg + (size_t)s * kMaxSeg + g, o);
-                    __threadfence();             // the segment (record and chunk partials) before it is counted
-                    last = atomicAdd(&sc.done[s], 1) == nseg - 1;
-                    if (last && n_todo < kTodo) { todo[n_todo] = s; n_todo = n_todo + 1; last = 0; }
-                }
-                last = __shfl_sync(0xffffffffu, last, 0);
-                if (last) {                      // queue full: finish at once
-                    __threadfence();
-                    finish_row<DT, FEATURES>(p, st, sc, a, s, nseg, lane);
-                }
+            last = __shfl_sync(0xffffffffu, last, 0);
+            if (last) {                      // queue full: finish at once
+                __threadfence();
+                finish_row<DT, FEATURES>(p, st, sc, a, s, nseg, lane);
             }
         }
-        __syncwarp();
-        // (the drain below needs the producer's final counts: after the CTA-wide barrier)
-        __syncthreads();
-        cons.drain(feed, warp);
-        // the rows this CTA completed, one warp each; their other segments were published before they were counted
-        if (n_todo > 0) __threadfence();
-        for (int j = warp; j < n_todo; j += kWarps) finish_row<DT, FEATURES>(p, st, sc, a, todo[j], nseg, lane);
-        return;
     }
-    __syncthreads();                             // producer warp: pairs with the folding warps' barrier above
+    __syncthreads();
+    // the rows this CTA completed, one warp each; their other segments were published before they were counted
+    if (n_todo > 0) __threadfence();
+    for (int j = warp; j < n_todo; j += kWarps) finish_row<DT, FEATURES>(p, st, sc, a, todo[j], nseg, lane);
 }
 
 // ============================================================================================
@@ -420,7 +377,7 @@ __device__ __forceinline__ int owner_locate(const WalkShared* sh, int which, int
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, kResident)
 k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
 {
     constexpr int ESZ = Elem<DT>::BYTES;
