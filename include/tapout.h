@@ -50,7 +50,9 @@ typedef enum {
     TAPOUT_E_ALIGNMENT = -3,    /* a logits pointer or stride is not 16-byte aligned    */
     TAPOUT_E_CUDA = -4,         /* a CUDA runtime call failed (tapout_last_cuda_error)  */
     TAPOUT_E_ALLOC = -5,        /* out of host or device memory                         */
-    TAPOUT_E_UNSUPPORTED = -6   /* valid request this build does not implement          */
+    TAPOUT_E_UNSUPPORTED = -6,  /* valid request this build does not implement          */
+    TAPOUT_E_TOO_LARGE = -7     /* more rows or a wider vocabulary than the built-in scratch of
+                                   tapout_row_stats_static holds                          */
 } tapout_error;
 
 /* Bandit algorithm (Section 3.3) and action granularity (Section 3.1). */
@@ -212,6 +214,34 @@ int tapout_round_host(tapout_t* h, const void* draft_logits, const void* target_
  */
 int tapout_row_stats(tapout_t* h, const void* logits, int n_rows, int64_t row_stride, double inv_temp,
                      float* out_features);
+
+/*
+ * No counterpart in the paper: a convenience of this library.  The same features as
+ * tapout_row_stats, for callers that must not allocate device memory: a serving loop that has
+ * handed the whole memory budget to its own pool, a component that runs where the implicit
+ * device-wide synchronisation of an allocation would stall other streams, or code that may
+ * not create a handle at all (tapout_create allocates).  No handle is needed and nothing is
+ * allocated or freed, by this library or through any allocating routine: the intermediate
+ * results live in one fixed array that is part of the loaded library image (about 330 KB on
+ * every GPU that loads it, held until the process exits).
+ *   logits       : device, n_rows rows of vocab elements, row_stride elements apart
+ *                  (16-byte aligned base, stride a multiple of 16 bytes)
+ *   dtype        : TAPOUT_DTYPE_FP32 or TAPOUT_DTYPE_BF16
+ *   out_features : device float [n_rows][6], as for tapout_row_stats
+ *   stream       : a cudaStream_t (as void*), may be NULL for the default stream
+ * Limits: n_rows <= TAPOUT_STATIC_MAX_ROWS and vocab <= TAPOUT_STATIC_MAX_VOCAB, otherwise
+ * TAPOUT_E_TOO_LARGE and nothing is launched.
+ * The first call on each device looks up the device address of the array (with that device
+ * current) and reads the device's SM count; make that first call outside any stream capture.
+ * Every call on a device uses the same array and finds in it whatever the call before left;
+ * the few counters that must start at zero are cleared at the start of each call, on `stream`.
+ * Two calls whose kernels can overlap on the GPU (different streams, no ordering between them)
+ * race on the array: order them yourself.
+ */
+#define TAPOUT_STATIC_MAX_ROWS 64
+#define TAPOUT_STATIC_MAX_VOCAB 262144
+int tapout_row_stats_static(const void* logits, int n_rows, int vocab, int64_t row_stride, int dtype,
+                            double inv_temp, float* out_features, void* stream);
 
 /*
  * State: bandit statistics, AdaEDL state and the current round's bookkeeping in

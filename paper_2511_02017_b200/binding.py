@@ -12,7 +12,8 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libtapout.so")
 
-OK, E_INVALID_ARG, E_BAD_STATE, E_ALIGNMENT, E_CUDA, E_ALLOC, E_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
+OK, E_INVALID_ARG, E_BAD_STATE, E_ALIGNMENT, E_CUDA, E_ALLOC, E_UNSUPPORTED, E_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6, -7
+STATIC_MAX_ROWS, STATIC_MAX_VOCAB = 64, 262144
 POLICY_UCB1, POLICY_TS, POLICY_UCB_TUNED = 0, 1, 2
 LEVEL_SEQ, LEVEL_TOKEN = 0, 1
 DTYPE_FP32, DTYPE_BF16 = 0, 1
@@ -36,7 +37,7 @@ EXPORTS = [
     "tapout_strerror", "tapout_last_cuda_error", "tapout_create", "tapout_destroy", "tapout_set_stream",
     "tapout_set_param_f64", "tapout_set_param_i64", "tapout_get_param_f64", "tapout_get_param_i64",
     "tapout_set_arms", "tapout_draft_step", "tapout_verify", "tapout_update", "tapout_round_host",
-    "tapout_row_stats", "tapout_state_bytes", "tapout_state_field", "tapout_get_state", "tapout_set_state",
+    "tapout_row_stats", "tapout_row_stats_static", "tapout_state_bytes", "tapout_state_field", "tapout_get_state", "tapout_set_state",
     "tapout_get_round", "tapout_set_round", "tapout_get_status", "tapout_get_profile", "tapout_get_launch_count",
 ]
 
@@ -87,6 +88,7 @@ def load():
     L.tapout_update.argtypes = [vp]
     L.tapout_round_host.argtypes = [vp, vp, vp, vp, vp, vp]
     L.tapout_row_stats.argtypes = [vp, vp, i32, i64, dbl, vp]
+    L.tapout_row_stats_static.argtypes = [vp, i32, i32, i64, i32, dbl, vp, vp]
     L.tapout_state_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
     L.tapout_state_field.argtypes = [vp, C.c_char_p, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     L.tapout_get_state.argtypes = [vp, vp]
@@ -108,6 +110,17 @@ def _dev_ptr(t, dtype=None):
     if dtype is not None and t.dtype != dtype:
         raise TypeError("expected dtype %s, got %s" % (dtype, t.dtype))
     return C.c_void_p(t.data_ptr())
+
+
+def row_stats_static(logits, n_rows, vocab, row_stride, dtype, inv_temp, out_features, stream=None):
+    """tapout_row_stats_static: features of up to STATIC_MAX_ROWS rows without a handle and without any
+    allocation (the scratch is a fixed array inside the library).  Raises TapoutError on a bad size."""
+    L = load()
+    ptr = stream.cuda_stream if isinstance(stream, torch.cuda.Stream) else int(stream or 0)
+    rc = L.tapout_row_stats_static(_dev_ptr(logits), n_rows, vocab, row_stride, dtype, float(inv_temp),
+                                   _dev_ptr(out_features, torch.float32), C.c_void_p(ptr))
+    if rc != OK:
+        raise TapoutError(rc, "tapout_row_stats_static")
 
 
 class Tapout:

@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -289,6 +290,7 @@ const char* tapout_strerror(int code) {
     case TAPOUT_E_CUDA: return "CUDA runtime error";
     case TAPOUT_E_ALLOC: return "out of memory";
     case TAPOUT_E_UNSUPPORTED: return "not supported";
+    case TAPOUT_E_TOO_LARGE: return "too many rows or too wide a vocabulary for the built-in scratch array";
     default: return "unknown error";
     }
 }
@@ -575,6 +577,85 @@ int tapout_row_stats(tapout_t* h, const void* logits, int n_rows, int64_t row_st
     if (h->p.dtype == DT_BF16) k_draft_step<DT_BF16, true><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->st, h->sc, a);
     else k_draft_step<DT_FP32, true><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->st, h->sc, a);
     TP_LAUNCHED(h);
+    return TAPOUT_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free row statistics: the scratch of the feature pass in a fixed array of the library image.
+// Layout (bytes): segment records [rows][kMaxSeg], chunk partials [rows][chunks], per-row counters.
+namespace {
+constexpr int kStaticMaxChunks = TAPOUT_STATIC_MAX_VOCAB / chunk_elems<DT_FP32>();     // fp32 chunks are the shorter ones
+constexpr size_t kStaticSegBytes = sizeof(SegRec) * TAPOUT_STATIC_MAX_ROWS * kMaxSeg;
+constexpr size_t kStaticCdfBytes = sizeof(float2) * (size_t)TAPOUT_STATIC_MAX_ROWS * kStaticMaxChunks;
+constexpr size_t kStaticDoneBytes = sizeof(int32_t) * TAPOUT_STATIC_MAX_ROWS;
+constexpr size_t kStaticBytes = kStaticSegBytes + kStaticCdfBytes + kStaticDoneBytes;
+}  // namespace
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+struct StaticDev { bool ready; char* base; int n_sm; };
+StaticDev g_static_dev[kMaxDevices];
+std::mutex g_static_mutex;
+
+// Device address of the array and SM count of the current device, looked up once per device.
+int static_setup(int dev, StaticDev* out) {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDev& d = g_static_dev[dev];
+    if (!d.ready) {
+        void* ptr = nullptr;
+        // in host code the array's name only stands for the symbol: its device address has to be asked for
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) { cudaGetLastError(); return TAPOUT_E_CUDA; }
+        int n_sm = 0;
+        if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 1) {
+            cudaGetLastError();
+            return TAPOUT_E_CUDA;
+        }
+        d.base = static_cast<char*>(ptr);
+        d.n_sm = n_sm;
+        d.ready = true;
+    }
+    *out = d;
+    return TAPOUT_OK;
+}
+}  // namespace
+
+int tapout_row_stats_static(const void* logits, int n_rows, int vocab, int64_t row_stride, int dtype, double inv_temp,
+                            float* out_features, void* stream) {
+    if (!logits || !out_features || n_rows < 1 || vocab < 2) return TAPOUT_E_INVALID_ARG;
+    if (dtype != DT_FP32 && dtype != DT_BF16) return TAPOUT_E_INVALID_ARG;
+    if (!(inv_temp > 0.0) || !((float)inv_temp < 1e30f)) return TAPOUT_E_INVALID_ARG;
+    if (n_rows > TAPOUT_STATIC_MAX_ROWS || vocab > TAPOUT_STATIC_MAX_VOCAB) return TAPOUT_E_TOO_LARGE;
+    const int esz = dtype == DT_BF16 ? 2 : 4;
+    if (row_stride < vocab) return TAPOUT_E_INVALID_ARG;
+    if (!aligned16(logits) || (row_stride * esz) % 16 != 0) return TAPOUT_E_ALIGNMENT;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return TAPOUT_E_CUDA; }
+    if (dev < 0 || dev >= kMaxDevices) return TAPOUT_E_UNSUPPORTED;
+    StaticDev d;
+    { int rc = static_setup(dev, &d); if (rc != TAPOUT_OK) return rc; }
+
+    Params p = {};
+    p.S = n_rows; p.V = vocab; p.K = 1; p.A = 1; p.P = 1; p.dtype = dtype;
+    const int CH = dtype == DT_BF16 ? chunk_elems<DT_BF16>() : chunk_elems<DT_FP32>();
+    p.NC = (vocab + CH - 1) / CH;                               // <= kStaticMaxChunks by the vocabulary limit
+    p.nseg = 0;
+    State st = {};                                              // the feature pass touches no round state
+    Scratch sc = {};
+    sc.seg = reinterpret_cast<SegRec*>(d.base);
+    sc.cdf = reinterpret_cast<float2*>(d.base + kStaticSegBytes);
+    sc.done = reinterpret_cast<int32_t*>(d.base + kStaticSegBytes + kStaticCdfBytes);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    // the per-row segment counters are the only part that has to start at zero
+    if (cudaMemsetAsync(sc.done, 0, kStaticDoneBytes, s) != cudaSuccess) { cudaGetLastError(); return TAPOUT_E_CUDA; }
+    StepArgs a = {};
+    a.logits = logits; a.row_stride = row_stride; a.n_fixed = n_rows;
+    a.c = c_of((float)inv_temp); a.inv_T = (float)inv_temp; a.tok_stride = 1; a.out_feat = out_features;
+    const int grid = d.n_sm * kResident;
+    if (dtype == DT_BF16) k_draft_step<DT_BF16, true><<<grid, kThreads, 0, s>>>(p, st, sc, a);
+    else k_draft_step<DT_FP32, true><<<grid, kThreads, 0, s>>>(p, st, sc, a);
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return TAPOUT_E_CUDA; }
     return TAPOUT_OK;
 }
 

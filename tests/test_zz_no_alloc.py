@@ -1,0 +1,93 @@
+"""tapout_row_stats_static, the entry point for callers that may not allocate device memory (a server
+whose memory pool owns the whole budget, code that cannot afford the device-wide stall of an allocation,
+code that has no handle because creating one allocates).  Its intermediate results live in a fixed array
+inside the library, shared by all calls, so the check is: same features as the handle-based
+tapout_row_stats on the same rows, on two calls in a row (the second call finds the first one's leftovers
+in the array), and sizes beyond the array are refused before anything is launched.
+
+Collected last on purpose (file name): a run that stops at the first failure has then already run every
+other test."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2511_02017_b200 import binding as tp
+from tests.lockstep import FEAT_FLOOR, FEAT_RTOL
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _rows(n, V, Vs, dtype, seed):
+    g = torch.Generator(device="cpu")
+    g.manual_seed(seed)
+    x = torch.randn((n, Vs), generator=g) * 3.0
+    x[:, :V] -= 1.1 * torch.log1p(torch.rand((n, V), generator=g) * V)
+    x[0, 5] = 9.0                                   # a clear maximum
+    x[1, 7] = x[1, 900] = 11.0                      # a duplicated maximum
+    x[2, ::3] = float("-inf")                       # masked tokens
+    x[3, 10] = float("nan")                         # unusable row
+    return x.to(dtype).to(DEV)
+
+
+def _close(a, b):
+    a, b = a.astype(np.float64), b.astype(np.float64)
+    nan_a, nan_b = np.isnan(a[:, :5]).all(axis=1), np.isnan(b[:, :5]).all(axis=1)
+    assert np.array_equal(nan_a, nan_b)
+    ok = ~nan_a
+    err = np.abs(a[ok, :5] - b[ok, :5]) / np.maximum(np.abs(b[ok, :5]), FEAT_FLOOR)
+    assert err.max() <= FEAT_RTOL, err.max()
+    assert np.array_equal(a[:, 5], b[:, 5])
+
+
+@pytest.mark.parametrize("dtype,code", [(torch.bfloat16, tp.DTYPE_BF16), (torch.float32, tp.DTYPE_FP32)])
+def test_static_scratch_matches_handle_path_twice_in_a_row(dtype, code):
+    n, V, Vs = 40, 9003, 9008
+    h = tp.Tapout(n, V, 2, 1, tp.POLICY_UCB1, tp.LEVEL_SEQ, dtype=code)
+    for call, (seed, inv_T) in enumerate([(1, 1.0), (2, 1.0 / 0.7)]):      # second call: other rows, other scale
+        x = _rows(n, V, Vs, dtype, seed)
+        want = torch.zeros((n, 6), dtype=torch.float32, device=DEV)
+        h.row_stats(x, n, Vs, inv_T, want)
+        got = torch.full((n, 6), -7.0, dtype=torch.float32, device=DEV)
+        tp.row_stats_static(x, n, V, Vs, code, inv_T, got)
+        torch.cuda.synchronize()
+        _close(got.cpu().numpy(), want.cpu().numpy())
+        # fewer rows than the call before: what the larger call left in the array must not leak in
+        got2 = torch.full((5, 6), -7.0, dtype=torch.float32, device=DEV)
+        tp.row_stats_static(x, 5, V, Vs, code, inv_T, got2)
+        torch.cuda.synchronize()
+        _close(got2.cpu().numpy(), want.cpu().numpy()[:5])
+    h.destroy()
+
+
+def test_static_scratch_on_a_side_stream():
+    n, V = 8, 4096
+    x = _rows(n, V, V, torch.bfloat16, 3)
+    out_a = torch.zeros((n, 6), dtype=torch.float32, device=DEV)
+    out_b = torch.zeros((n, 6), dtype=torch.float32, device=DEV)
+    tp.row_stats_static(x, n, V, V, tp.DTYPE_BF16, 1.0, out_a)
+    torch.cuda.synchronize()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        tp.row_stats_static(x, n, V, V, tp.DTYPE_BF16, 1.0, out_b, stream=s)
+    s.synchronize()
+    assert torch.equal(out_a.isnan(), out_b.isnan())
+    assert torch.equal(out_a.nan_to_num(), out_b.nan_to_num())
+
+
+def test_sizes_beyond_the_fixed_array_are_refused():
+    L = tp.load()
+    x = torch.zeros((2, 4096), dtype=torch.bfloat16, device=DEV)
+    out = torch.zeros((2, 6), dtype=torch.float32, device=DEV)
+    args = lambda n, V, stride: (C.c_void_p(x.data_ptr()), n, V, stride, tp.DTYPE_BF16, 1.0,
+                                 C.c_void_p(out.data_ptr()), None)
+    assert L.tapout_row_stats_static(*args(tp.STATIC_MAX_ROWS + 1, 4096, 4096)) == tp.E_TOO_LARGE
+    assert L.tapout_row_stats_static(*args(2, tp.STATIC_MAX_VOCAB + 8, tp.STATIC_MAX_VOCAB + 8)) == tp.E_TOO_LARGE
+    assert L.tapout_row_stats_static(*args(0, 4096, 4096)) == tp.E_INVALID_ARG
+    assert L.tapout_row_stats_static(*args(2, 4096, 4090)) == tp.E_INVALID_ARG          # stride shorter than a row
+    assert L.tapout_row_stats_static(*args(2, 4090, 4091)) == tp.E_ALIGNMENT
+    assert L.tapout_row_stats_static(None, 2, 4096, 4096, tp.DTYPE_BF16, 1.0, C.c_void_p(out.data_ptr()), None) == tp.E_INVALID_ARG
+    assert L.tapout_strerror(tp.E_TOO_LARGE) not in (b"ok", b"unknown error")
+    torch.cuda.synchronize()
