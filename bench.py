@@ -214,30 +214,28 @@ def bench_ours(args):
     rows_all, ms_all = aggregate(rows, ms, world, backend_ready)
     value = rows_all / (ms_all * 1e-3)
 
-    # ---- per-kernel device time (separate pass, same steps, events around the two streaming kernels)
+    # ---- per-kernel device time (separate pass, same steps, event intervals per kernel class)
     dev.set_param("profile", 1)
-    for k in range(4):
+    for k in range(3):
         dev.get_profile(k, reset=True)
     sp0 = dev.get_status()
     prof_steps = min(args.steps, 64)
     for r in range(prof_steps):
         step(args.warmup + args.steps + r)
     torch.cuda.synchronize()
-    prof = [dev.get_profile(k, reset=True) for k in range(4)]
+    prof = [dev.get_profile(k, reset=True) for k in range(3)]
     sp1 = dev.get_status()
     dev.set_param("profile", 0)
     peak, peak_src = measured_peaks()
     row_bytes = w.row_bytes
     d_rows = sp1["rows_draft"] - sp0["rows_draft"]
-    d0_rows = min(d_rows, prof_steps * S)                 # every sequence drafts at position 0
     v_rows = (sp1["rows_target"] - sp0["rows_target"]) + (sp1["rows_residual"] - sp0["rows_residual"])
 
     def kinfo(k, rows_k):
         ms_k, n_k = prof[k]
         return {"launches": n_k, "ms_total": ms_k, "alg_bytes": rows_k * row_bytes,
                 "gbs": rows_k * row_bytes / (ms_k * 1e-3) / 1e9 if ms_k > 0 else None}
-    kernels = {"k_draft_step@pos0": kinfo(0, d0_rows), "k_verify_walk": kinfo(1, v_rows),
-               "k_draft_step@pos>0": kinfo(2, d_rows - d0_rows), "k_update": kinfo(3, 0)}
+    kernels = {"k_draft_step": kinfo(0, d_rows), "k_verify_walk": kinfo(1, v_rows), "k_update": kinfo(2, 0)}
     dom = max(kernels, key=lambda k: kernels[k]["ms_total"])
     achieved = kernels[dom]["gbs"] or 0.0
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -350,8 +348,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample-seqs", type=int, default=256)
-    ap.add_argument("--cpu-sample-rounds", type=int, default=4)
+    ap.add_argument("--cpu-sample-seqs", type=int, default=512)
+    ap.add_argument("--cpu-sample-rounds", type=int, default=72)
     ap.add_argument("--ref-sample-seqs", type=int, default=32)
     ap.add_argument("--n-seq", type=int, default=0, help="override the batch size (profiling captures)")
     ap.add_argument("--row-segments", type=int, default=0, help="CTAs per draft row (0 = library default)")

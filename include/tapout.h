@@ -273,10 +273,11 @@ int tapout_get_status(tapout_t* h, uint64_t* bits, uint64_t* rows_draft, uint64_
                       uint64_t* rows_residual);
 
 /*
- * With TAPOUT_P_PROFILE = 1 every kernel launch of the round is bracketed by CUDA events on the
- * handle's stream, in four classes: 0 draft step at position 0, 1 verification walk, 2 draft steps at
- * later positions, 3 update.  Synchronises, returns the summed device time in milliseconds and the
- * number of launches of that class since the last reset; reset != 0 clears both.
+ * With TAPOUT_P_PROFILE = 1 the kernels of a round are timed with CUDA events on the handle's
+ * stream, in three classes: 0 the draft steps of a round (one interval from the first step's launch
+ * to the call of tapout_verify, so the gaps between the steps count), 1 the verification walk,
+ * 2 the update.  Synchronises, returns the summed device time in milliseconds and the number of
+ * kernel launches of that class since the last reset; reset != 0 clears both.
  */
 int tapout_get_profile(tapout_t* h, int kernel, double* ms, uint64_t* launches, int reset);
 

@@ -23,7 +23,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace
 
-constexpr int kProf = 4;   // timed launch classes: draft step at position 0, verify, draft steps at later positions, update
+constexpr int kProf = 3;   // timed launch classes: the draft steps of a round, verify, update
 
 struct tapout {
     Params p{};
@@ -58,7 +58,7 @@ struct tapout {
     bool profile = false;
     std::vector<cudaEvent_t> ev[kProf];  // start/stop pairs not yet read back
     double prof_ms[kProf] = {};
-    uint64_t prof_n[kProf] = {};
+    uint64_t prof_n[kProf] = {};        // launches of the class since the last reset
 };
 
 namespace {
@@ -186,7 +186,6 @@ int drain_profile(tapout* h, int k) {
         cudaEventDestroy(h->ev[k][i + 1]);
         if (e != cudaSuccess) { h->ev[k].clear(); return fail_cuda(h, e, "profile events"); }
         h->prof_ms[k] += ms;
-        h->prof_n[k] += 1;
     }
     h->ev[k].clear();
     return TAPOUT_OK;
@@ -200,6 +199,31 @@ int profile_mark(tapout* h, int k) {
     h->ev[k].push_back(e);
     TP_CUDA(h, cudaEventRecord(e, h->stream));
     return TAPOUT_OK;
+}
+
+// Launch with programmatic stream serialization: the kernel may be scheduled while its predecessor in the
+// stream drains; every kernel of the round waits (pdl_wait) before it touches anything the predecessor
+// wrote.  cluster > 1 adds the cluster dimension.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t stream,
+                           int cluster, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[2];
+    int n = 0;
+    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cluster > 0) {
+        at[n].id = cudaLaunchAttributeClusterDimension;
+        at[n].val.clusterDim.x = (unsigned)cluster; at[n].val.clusterDim.y = 1; at[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = at; cfg.numAttrs = (unsigned)n;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 StepArgs step_args(const tapout* h, const void* logits, int64_t stride, float c) {
@@ -219,28 +243,21 @@ int draft_step_impl(tapout* h, const void* logits, int64_t stride, int32_t* out_
     if (h->pos == 0 && !h->arms_ready) { int rc = begin_round_now(h, 0); if (rc) return rc; }
     StepArgs a = step_args(h, logits, stride, c_of(h->p.inv_Tq));
     a.out_token = out_token; a.tok_stride = tok_stride; a.out_continue = out_continue;
-    const int pk = h->pos == 0 ? 0 : 2;
-    { int rc = profile_mark(h, pk); if (rc) return rc; }
-    if (h->p.dtype == DT_BF16) k_draft_step<DT_BF16, false><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->st, h->sc, a);
-    else k_draft_step<DT_FP32, false><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->st, h->sc, a);
+    // one event pair per round for all draft steps: opened here, closed when verify is called
+    if (h->pos == 0) { int rc = profile_mark(h, 0); if (rc) return rc; }
+    if (h->profile) h->prof_n[0] += 1;
+    TP_CUDA(h, h->p.dtype == DT_BF16
+                   ? launch_chained(k_draft_step<DT_BF16, false>, h->grid_rows, kThreads, 0, h->stream, 0, h->p, h->st, h->sc, a)
+                   : launch_chained(k_draft_step<DT_FP32, false>, h->grid_rows, kThreads, 0, h->stream, 0, h->p, h->st, h->sc, a));
     TP_LAUNCHED(h);
-    { int rc = profile_mark(h, pk); if (rc) return rc; }
     h->pos += 1;
     return TAPOUT_OK;
 }
 
 template <int DT>
 cudaError_t launch_walk(tapout* h, const WalkArgs& a) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)h->p.S * (unsigned)h->cluster, 1, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = h->walk_smem;
-    cfg.stream = h->stream;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = (unsigned)h->cluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_verify_walk<DT>, h->p, h->st, h->sc, a);
+    return launch_chained(k_verify_walk<DT>, (unsigned)h->p.S * (unsigned)h->cluster, kThreads, h->walk_smem, h->stream,
+                          h->cluster, h->p, h->st, h->sc, a);
 }
 
 int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const void* pl, int64_t p_seq, int64_t p_pos,
@@ -255,10 +272,12 @@ int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const vo
     a.toks = toks; a.slot = h->pos % 3; a.round = h->round;
     a.cq = c_of(h->p.inv_Tq); a.cp = c_of(h->p.inv_Tp);
     a.out_acc = out_acc; a.out_next = out_next;
+    if (h->ev[0].size() % 2 == 1) { int rc = profile_mark(h, 0); if (rc) return rc; }
     { int rc = profile_mark(h, 1); if (rc) return rc; }
     TP_CUDA(h, h->p.dtype == DT_BF16 ? launch_walk<DT_BF16>(h, a) : launch_walk<DT_FP32>(h, a));
     TP_LAUNCHED(h);
     { int rc = profile_mark(h, 1); if (rc) return rc; }
+    if (h->profile) h->prof_n[1] += 1;
     h->verified = true;
     return TAPOUT_OK;
 }
@@ -266,10 +285,11 @@ int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const vo
 int update_impl(tapout* h) {
     if (!h) return TAPOUT_E_INVALID_ARG;
     if (!h->verified) return TAPOUT_E_BAD_STATE;
-    { int rc = profile_mark(h, 3); if (rc) return rc; }
-    k_update<<<(h->p.S + 3) / 4, 128, 0, h->stream>>>(h->p, h->st, h->sc, h->round + 1);
+    { int rc = profile_mark(h, 2); if (rc) return rc; }
+    TP_CUDA(h, launch_chained(k_update, (unsigned)(h->p.S + 3) / 4, 128, 0, h->stream, 0, h->p, h->st, h->sc, h->round + 1));
     TP_LAUNCHED(h);
-    { int rc = profile_mark(h, 3); if (rc) return rc; }
+    { int rc = profile_mark(h, 2); if (rc) return rc; }
+    if (h->profile) h->prof_n[2] += 1;
     h->round += 1;
     h->pos = 0;
     h->verified = false;

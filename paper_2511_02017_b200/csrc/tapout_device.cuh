@@ -68,6 +68,13 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start
+// while its predecessor in the stream is still draining.  pdl_wait() returns once the predecessor has
+// completed and its writes are visible: nothing it wrote or reads may be touched before.
+// pdl_trigger() lets the successor's CTAs be scheduled as soon as room frees up.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
 
 // Warp maximum through the integer reduction unit: floats map monotonically to ints.

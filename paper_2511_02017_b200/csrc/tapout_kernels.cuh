@@ -230,6 +230,8 @@ k_draft_step(Params p, State st, Scratch sc, StepArgs a)
     __shared__ int n_todo;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) n_todo = 0;
+    pdl_trigger();
+    pdl_wait();
     const int n_rows = FEATURES ? a.n_fixed : sc.count[a.slot];
     const int32_t* list = sc.list + (size_t)a.slot * p.S;
     if (!FEATURES) {
@@ -389,6 +391,8 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
     const int cid = blockIdx.x / CS;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
+    pdl_trigger();
+    pdl_wait();
     // longest drafts first: sequences still drafting, then the stopped ones, last stopped first
     const int n_act = sc.count[a.slot];
     const int s = (cid < n_act) ? sc.list[(size_t)a.slot * p.S + cid] : sc.stopped[p.S - 1 - cid];
@@ -617,6 +621,8 @@ k_update(Params p, State st, Scratch sc, uint32_t next_round)
     __shared__ uint32_t hist[4][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int s = blockIdx.x * 4 + warp;
+    pdl_trigger();
+    pdl_wait();
     if (s >= p.S) return;
     if (lane == 0) {
         const int n = st.n_drafted[s], a = st.accept_len[s];
@@ -659,6 +665,8 @@ k_begin_round(Params p, State st, Scratch sc, uint32_t round, int reset_adaedl)
     __shared__ uint32_t hist[4][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int s = blockIdx.x * 4 + warp;
+    pdl_trigger();
+    pdl_wait();
     if (s >= p.S) return;
     if (reset_adaedl && lane == 0) { st.lambda[s] = p.ada_lambda0; st.acc_rate[s] = p.ada_acc0; }
     __syncwarp();
