@@ -125,11 +125,7 @@ def aggregate(rows_local, ms_local, world, backend_ready):
 
 # ----------------------------------------------------------------------------------------------
 def run_round(dev, w, draft, target, toks, cont, acc, nxt):
-    K = w.k_max
-    for i in range(K):
-        dev.draft_step(draft[:, i, :], toks[:, i], cont)
-    dev.verify(draft, target, toks, acc, nxt)
-    dev.update()
+    dev.round(draft, target, toks, cont, acc, nxt)
 
 
 def oracle_sample(w, draft, target, n_seq_sample, rounds, seq_offset=0):

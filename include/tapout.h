@@ -194,6 +194,22 @@ int tapout_verify(tapout_t* h, const void* draft_probs, const void* target_logit
 int tapout_update(tapout_t* h);
 
 /*
+ * Algorithm 1, one whole round with every tensor already on the device: k_max calls of
+ * tapout_draft_step (step i reads position i of draft_logits and writes column i of
+ * out_draft_tokens), tapout_verify and tapout_update, enqueued back to back on the handle's
+ * stream without synchronising.  Same kernels and results as the separate calls; it only saves
+ * the caller k_max + 2 trips through the boundary.  A sequence that has stopped gets -1 in the
+ * remaining columns of out_draft_tokens.
+ *   draft_logits  : device, [n_seq][k_max][vocab] (strides TAPOUT_P_Q_*)
+ *   target_logits : device, [n_seq][k_max+1][vocab] (strides TAPOUT_P_P_*)
+ *   out_draft_tokens : device, int32 [n_seq][k_max];  out_continue : device, uint8 [n_seq] (the
+ *                      last step's flags);  out_accept_len, out_next_token : device, int32 [n_seq]
+ * TAPOUT_E_BAD_STATE unless called between rounds.
+ */
+int tapout_round(tapout_t* h, const void* draft_logits, const void* target_logits, int32_t* out_draft_tokens,
+                 uint8_t* out_continue, int32_t* out_accept_len, int32_t* out_next_token);
+
+/*
  * One whole round from HOST memory: copies the round's logits to the device,
  * runs k_max draft steps, verify and update, and copies the results back.
  * Blocks until done.  Host arrays: draft_logits [n_seq][k_max][vocab],
@@ -222,7 +238,7 @@ int tapout_row_stats(tapout_t* h, const void* logits, int n_rows, int64_t row_st
  * device-wide synchronisation of an allocation would stall other streams, or code that may
  * not create a handle at all (tapout_create allocates).  No handle is needed and nothing is
  * allocated or freed, by this library or through any allocating routine: the intermediate
- * results live in one fixed array that is part of the loaded library image (about 330 KB on
+ * results live in one fixed array that is part of the loaded library image (about 400 KB on
  * every GPU that loads it, held until the process exits).
  *   logits       : device, n_rows rows of vocab elements, row_stride elements apart
  *                  (16-byte aligned base, stride a multiple of 16 bytes)

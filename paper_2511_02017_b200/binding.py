@@ -36,7 +36,7 @@ _INT_PARAMS = {"seed", "dtype", "seq_offset", "step_row_stride", "q_seq_stride",
 EXPORTS = [
     "tapout_strerror", "tapout_last_cuda_error", "tapout_create", "tapout_destroy", "tapout_set_stream",
     "tapout_set_param_f64", "tapout_set_param_i64", "tapout_get_param_f64", "tapout_get_param_i64",
-    "tapout_set_arms", "tapout_draft_step", "tapout_verify", "tapout_update", "tapout_round_host",
+    "tapout_set_arms", "tapout_draft_step", "tapout_verify", "tapout_update", "tapout_round", "tapout_round_host",
     "tapout_row_stats", "tapout_row_stats_static", "tapout_state_bytes", "tapout_state_field", "tapout_get_state", "tapout_set_state",
     "tapout_get_round", "tapout_set_round", "tapout_get_status", "tapout_get_profile", "tapout_get_launch_count",
 ]
@@ -86,6 +86,7 @@ def load():
     L.tapout_draft_step.argtypes = [vp, vp, vp, vp]
     L.tapout_verify.argtypes = [vp, vp, vp, vp, vp, vp]
     L.tapout_update.argtypes = [vp]
+    L.tapout_round.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.tapout_round_host.argtypes = [vp, vp, vp, vp, vp, vp]
     L.tapout_row_stats.argtypes = [vp, vp, i32, i64, dbl, vp]
     L.tapout_row_stats_static.argtypes = [vp, i32, i32, i64, i32, dbl, vp, vp]
@@ -206,6 +207,13 @@ class Tapout:
 
     def update(self):
         self._check(self.L.tapout_update(self.h), "tapout_update")
+
+    def round(self, draft_logits, target_logits, out_draft_tokens, out_continue, out_accept_len, out_next_token):
+        """tapout_round: the k_max draft steps, verify and update of one round on device tensors."""
+        self._check(self.L.tapout_round(self.h, _dev_ptr(draft_logits), _dev_ptr(target_logits),
+                                        _dev_ptr(out_draft_tokens, torch.int32), _dev_ptr(out_continue, torch.uint8),
+                                        _dev_ptr(out_accept_len, torch.int32), _dev_ptr(out_next_token, torch.int32)),
+                    "tapout_round")
 
     def round_host(self, draft_logits, target_logits, out_draft_tokens, out_accept_len, out_next_token):
         """All arguments are CPU tensors (pinned or not); blocks until the round is done."""

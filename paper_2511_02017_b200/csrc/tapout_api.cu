@@ -144,7 +144,7 @@ int setup_scratch(tapout* h) {
     const size_t o_seg = off;    off = align_up(off + sizeof(SegRec) * (size_t)p.S * kMaxSeg, 256);
     const size_t o_cdf = off;    off = align_up(off + sizeof(float2) * (size_t)p.S * p.NC, 256);
     const size_t o_list = off;   off = align_up(off + sizeof(int32_t) * 3 * (size_t)p.S, 256);
-    const size_t o_count = off;  off = align_up(off + sizeof(int32_t) * 4, 256);
+    const size_t o_count = off;  off = align_up(off + sizeof(int32_t) * 8, 256);
     const size_t o_stop = off;   off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
     const size_t o_next = off;   off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
     const size_t o_done = off;   off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
@@ -245,10 +245,16 @@ int draft_step_impl(tapout* h, const void* logits, int64_t stride, int32_t* out_
     a.out_token = out_token; a.tok_stride = tok_stride; a.out_continue = out_continue;
     // one event pair per round for all draft steps: opened here, closed when verify is called
     if (h->pos == 0) { int rc = profile_mark(h, 0); if (rc) return rc; }
-    if (h->profile) h->prof_n[0] += 1;
+    if (h->profile) h->prof_n[0] += 2;
+    const unsigned fin_grid = (unsigned)((h->p.S + 3) / 4);
+    const int n_warps = h->grid_rows * kWarps;
     TP_CUDA(h, h->p.dtype == DT_BF16
-                   ? launch_chained(k_draft_step<DT_BF16, false>, h->grid_rows, kThreads, 0, h->stream, 0, h->p, h->st, h->sc, a)
-                   : launch_chained(k_draft_step<DT_FP32, false>, h->grid_rows, kThreads, 0, h->stream, 0, h->p, h->st, h->sc, a));
+                   ? launch_chained(k_draft_stream<DT_BF16, false>, h->grid_rows, kThreads, 0, h->stream, 0, h->p, h->sc, a)
+                   : launch_chained(k_draft_stream<DT_FP32, false>, h->grid_rows, kThreads, 0, h->stream, 0, h->p, h->sc, a));
+    TP_LAUNCHED(h);
+    TP_CUDA(h, h->p.dtype == DT_BF16
+                   ? launch_chained(k_draft_finish<DT_BF16, false>, fin_grid, kFinishThreads, 0, h->stream, 0, h->p, h->st, h->sc, a, n_warps)
+                   : launch_chained(k_draft_finish<DT_FP32, false>, fin_grid, kFinishThreads, 0, h->stream, 0, h->p, h->st, h->sc, a, n_warps));
     TP_LAUNCHED(h);
     h->pos += 1;
     return TAPOUT_OK;
@@ -542,6 +548,23 @@ int tapout_verify(tapout_t* h, const void* draft_probs, const void* target_logit
 
 int tapout_update(tapout_t* h) { return update_impl(h); }
 
+int tapout_round(tapout_t* h, const void* draft_logits, const void* target_logits, int32_t* out_draft_tokens,
+                 uint8_t* out_continue, int32_t* out_accept_len, int32_t* out_next_token) {
+    if (!h || !draft_logits || !target_logits || !out_draft_tokens || !out_continue || !out_accept_len || !out_next_token)
+        return TAPOUT_E_INVALID_ARG;
+    if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
+    const size_t esz = elem_bytes(h);
+    for (int i = 0; i < h->p.K; ++i) {
+        const char* rows = static_cast<const char*>(draft_logits) + (size_t)i * (size_t)h->q_pos * esz;
+        int rc = draft_step_impl(h, rows, h->q_seq, out_draft_tokens + i, (int64_t)h->p.K, out_continue);
+        if (rc != TAPOUT_OK) return rc;
+    }
+    int rc = verify_impl(h, draft_logits, h->q_seq, h->q_pos, target_logits, h->p_seq, h->p_pos, out_draft_tokens,
+                         out_accept_len, out_next_token);
+    if (rc != TAPOUT_OK) return rc;
+    return update_impl(h);
+}
+
 int tapout_round_host(tapout_t* h, const void* draft_logits, const void* target_logits, int32_t* out_draft_tokens,
                       int32_t* out_accept_len, int32_t* out_next_token) {
     if (!h || !draft_logits || !target_logits || !out_draft_tokens || !out_accept_len || !out_next_token)
@@ -594,8 +617,16 @@ int tapout_row_stats(tapout_t* h, const void* logits, int n_rows, int64_t row_st
     if (!aligned16(logits) || !stride_ok(h, row_stride) || row_stride < h->p.V) return TAPOUT_E_ALIGNMENT;
     StepArgs a = step_args(h, logits, row_stride, c_of((float)inv_temp));
     a.n_fixed = n_rows; a.inv_T = (float)inv_temp; a.out_feat = out_features;
-    if (h->p.dtype == DT_BF16) k_draft_step<DT_BF16, true><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->st, h->sc, a);
-    else k_draft_step<DT_FP32, true><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->st, h->sc, a);
+    const int n_warps = h->grid_rows * kWarps;
+    if (h->p.dtype == DT_BF16) {
+        k_draft_stream<DT_BF16, true><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->sc, a);
+        TP_LAUNCHED(h);
+        k_draft_finish<DT_BF16, true><<<(n_rows + 3) / 4, kFinishThreads, 0, h->stream>>>(h->p, h->st, h->sc, a, n_warps);
+    } else {
+        k_draft_stream<DT_FP32, true><<<h->grid_rows, kThreads, 0, h->stream>>>(h->p, h->sc, a);
+        TP_LAUNCHED(h);
+        k_draft_finish<DT_FP32, true><<<(n_rows + 3) / 4, kFinishThreads, 0, h->stream>>>(h->p, h->st, h->sc, a, n_warps);
+    }
     TP_LAUNCHED(h);
     return TAPOUT_OK;
 }
@@ -607,7 +638,7 @@ namespace {
 constexpr int kStaticMaxChunks = TAPOUT_STATIC_MAX_VOCAB / chunk_elems<DT_FP32>();     // fp32 chunks are the shorter ones
 constexpr size_t kStaticSegBytes = sizeof(SegRec) * TAPOUT_STATIC_MAX_ROWS * kMaxSeg;
 constexpr size_t kStaticCdfBytes = sizeof(float2) * (size_t)TAPOUT_STATIC_MAX_ROWS * kStaticMaxChunks;
-constexpr size_t kStaticDoneBytes = sizeof(int32_t) * TAPOUT_STATIC_MAX_ROWS;
+constexpr size_t kStaticDoneBytes = sizeof(int32_t) * (TAPOUT_STATIC_MAX_ROWS + 8);    // per-row counters, then `count`
 constexpr size_t kStaticBytes = kStaticSegBytes + kStaticCdfBytes + kStaticDoneBytes;
 }  // namespace
 
@@ -666,15 +697,21 @@ int tapout_row_stats_static(const void* logits, int n_rows, int vocab, int64_t r
     sc.seg = reinterpret_cast<SegRec*>(d.base);
     sc.cdf = reinterpret_cast<float2*>(d.base + kStaticSegBytes);
     sc.done = reinterpret_cast<int32_t*>(d.base + kStaticSegBytes + kStaticCdfBytes);
+    sc.count = sc.done + TAPOUT_STATIC_MAX_ROWS;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    // the per-row segment counters are the only part that has to start at zero
+    // the per-row segment counters and the work ticket are the only part that has to start at zero
     if (cudaMemsetAsync(sc.done, 0, kStaticDoneBytes, s) != cudaSuccess) { cudaGetLastError(); return TAPOUT_E_CUDA; }
     StepArgs a = {};
     a.logits = logits; a.row_stride = row_stride; a.n_fixed = n_rows;
     a.c = c_of((float)inv_temp); a.inv_T = (float)inv_temp; a.tok_stride = 1; a.out_feat = out_features;
     const int grid = d.n_sm * kResident;
-    if (dtype == DT_BF16) k_draft_step<DT_BF16, true><<<grid, kThreads, 0, s>>>(p, st, sc, a);
-    else k_draft_step<DT_FP32, true><<<grid, kThreads, 0, s>>>(p, st, sc, a);
+    if (dtype == DT_BF16) {
+        k_draft_stream<DT_BF16, true><<<grid, kThreads, 0, s>>>(p, sc, a);
+        k_draft_finish<DT_BF16, true><<<(n_rows + 3) / 4, kFinishThreads, 0, s>>>(p, st, sc, a, grid * kWarps);
+    } else {
+        k_draft_stream<DT_FP32, true><<<grid, kThreads, 0, s>>>(p, sc, a);
+        k_draft_finish<DT_FP32, true><<<(n_rows + 3) / 4, kFinishThreads, 0, s>>>(p, st, sc, a, grid * kWarps);
+    }
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return TAPOUT_E_CUDA; }
     return TAPOUT_OK;
 }

@@ -14,7 +14,7 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kMaxArms = 16;
 constexpr int kFeat = 6;                 // m, lse, p1, p2, H, argmax
 constexpr int kVecPerLane = 4;           // 16-byte loads per lane and chunk -> 2 KB per warp chunk
-constexpr int kMaxSeg = 32;              // CTAs sharing one row (one lane per segment in the finish)
+constexpr int kMaxSeg = 64;              // warps sharing one draft row (two segment records per lane in the finish)
 constexpr double kLog2e = 1.4426950408889634074;
 constexpr double kLn2 = 0.6931471805599453094;
 
@@ -54,7 +54,8 @@ struct Scratch {
     SegRec* seg;                 // [S][kMaxSeg]
     float2* cdf;                 // [S][NC]: (reference logit, sum of 2^(z*c + k)) per chunk
     int32_t* list;               // [3][S] sequences drafting at position pos, in slot pos % 3
-    int32_t* count;              // [0..2] lengths of the three lists; [3] length of `stopped`
+    int32_t* count;              // [0..2] lengths of the three lists; [3] length of `stopped`; [4],[5] work tickets of
+                                 // the draft step by position parity; [6] work ticket of tapout_row_stats
     int32_t* stopped;            // [S] sequences in the order in which they stopped drafting this round
     int32_t* next_pos;           // [S] position the sequence drafts at next (stays put once it has stopped)
     int32_t* done;               // [S] segments of the sequence's current row already reduced
@@ -408,7 +409,6 @@ __device__ __forceinline__ double scaled_contrib(float2 p, float c, double mc) {
 
 struct RegCdf {
     float2 part[kRegPer];      // this lane's chunks: lane * per .. lane * per + per - 1
-    double con[kRegPer];       // their contributions to the row total, relative to the row maximum
     double lane_sum, incl, W;
     int per, NC;
 
@@ -426,17 +426,15 @@ struct RegCdf {
     __device__ __forceinline__ void scale(float c, double mc, int lane) {
         double ls = 0.0;
 #pragma unroll
-        for (int j = 0; j < kRegPer; ++j) {
-            con[j] = (j < per) ? scaled_contrib(part[j], c, mc) : 0.0;
-            ls += con[j];
-        }
+        for (int j = 0; j < kRegPer; ++j) ls += scaled_contrib(part[j], c, mc);
         lane_sum = ls;
         incl = warp_incl_scan_d(ls, lane);
         W = __shfl_sync(0xffffffffu, incl, 31);
     }
     // Chunk in which the running sum first exceeds tgt (if rounding leaves none, the last chunk with a
-    // positive contribution), tgt minus the sum before it, and the chunk's reference logit.
-    __device__ __forceinline__ int locate(double tgt, int lane, double& rem, float& ref) const {
+    // positive contribution), tgt minus the sum before it, and the chunk's reference logit.  The
+    // contributions are formed again rather than kept: registers are scarcer than arithmetic here.
+    __device__ __forceinline__ int locate(double tgt, int lane, float c, double mc, double& rem, float& ref) const {
         const unsigned over = __ballot_sync(0xffffffffu, incl > tgt);
         const unsigned pos = __ballot_sync(0xffffffffu, lane_sum > 0.0);
         rem = 0.0; ref = 0.f;
@@ -450,7 +448,7 @@ struct RegCdf {
         float r_pick = 0.f, r_last = 0.f;
 #pragma unroll
         for (int j = 0; j < kRegPer; ++j) {
-            const double x = con[j];
+            const double x = scaled_contrib(part[j], c, mc);
             if (x > 0.0) { last_pos = j; before_last = run; r_last = part[j].x; }
             if (pick < 0 && run + x > tgt) { pick = j; before = run; r_pick = part[j].x; }
             run += x;
@@ -494,15 +492,17 @@ __device__ __forceinline__ float lane_block_elem(const uint4 (&v)[4], int k, int
     return idx < V ? z : neg_inf();
 }
 
-// Token inside one chunk.  Lane l owns the EPL consecutive tokens starting at first_token (its own); w
-// holds their weights (>= 0) exactly as the streaming pass formed them, t is the target inside the chunk
-// in the same units.  First token whose running sum exceeds t; if rounding leaves none, the last token
-// with positive weight.  Sums run in double so that the order of additions cannot matter.
-template <int EPL>
-__device__ __forceinline__ int pick_in_block(const float (&w)[EPL], int first_token, double t, int lane) {
+// Token inside one chunk.  Lane l owns the EPL consecutive tokens starting at first_token (its own);
+// weight(k) gives the weight (>= 0) of its k-th token exactly as the streaming pass formed it, t is the
+// target inside the chunk in the same units.  First token whose running sum exceeds t; if rounding
+// leaves none, the last token with positive weight.  Sums run in double so that the order of additions
+// cannot matter.  The weights are formed twice (once for the lane totals, once for the walk inside the
+// chosen lane) instead of being kept in an array of registers.
+template <int EPL, typename Weight>
+__device__ __forceinline__ int pick_in_block(Weight weight, int first_token, double t, int lane) {
     double sum = 0.0;
 #pragma unroll
-    for (int k = 0; k < EPL; ++k) sum += (double)w[k];
+    for (int k = 0; k < EPL; ++k) sum += (double)weight(k);
     const double incl = warp_incl_scan_d(sum, lane);
     const unsigned over = __ballot_sync(0xffffffffu, incl > t);
     const unsigned pos = __ballot_sync(0xffffffffu, sum > 0.0);
@@ -513,16 +513,14 @@ __device__ __forceinline__ int pick_in_block(const float (&w)[EPL], int first_to
     const double tl = t - (incl - sum);
     double run = 0.0;
     int pick = -1, last_pos = -1;
-    if (lane == L) {
 #pragma unroll
-        for (int k = 0; k < EPL; ++k) {
-            const double x = (double)w[k];
-            if (x > 0.0) last_pos = k;
-            run += x;
-            if (pick < 0 && run > tl) pick = k;
-        }
-        if (pick < 0) pick = last_pos;
+    for (int k = 0; k < EPL; ++k) {
+        const double x = (double)weight(k);
+        if (x > 0.0) last_pos = k;
+        run += x;
+        if (pick < 0 && run > tl) pick = k;
     }
+    if (pick < 0) pick = last_pos;
     return __shfl_sync(0xffffffffu, first_token + pick, L);
 }
 
@@ -531,10 +529,7 @@ template <int DT>
 __device__ __forceinline__ int pick_softmax_block(const uint4 (&v)[4], int V, int chunk, float c, float k, double t, int lane) {
     constexpr int EPL = chunk_elems<DT>() / 32;
     const int e0 = chunk * chunk_elems<DT>() + lane * EPL;
-    float w[EPL];
-#pragma unroll
-    for (int j = 0; j < EPL; ++j) w[j] = ex2_approx(fmaf(lane_block_elem<DT>(v, j, e0 + j, V), c, k));
-    return pick_in_block<EPL>(w, e0, t, lane);
+    return pick_in_block<EPL>([&](int j) { return ex2_approx(fmaf(lane_block_elem<DT>(v, j, e0 + j, V), c, k)); }, e0, t, lane);
 }
 
 template <int DT>
@@ -553,14 +548,11 @@ __device__ __forceinline__ int pick_residual(const void* prow, const void* qrow,
     uint4 vp[4], vq[4];
     load_lane_block<DT>(prow, V, chunk, lane, vp);
     load_lane_block<DT>(qrow, V, chunk, lane, vq);
-    float w[EPL];
-#pragma unroll
-    for (int j = 0; j < EPL; ++j) {
+    return pick_in_block<EPL>([&](int j) {
         const float wp = ex2_approx(fmaf(lane_block_elem<DT>(vp, j, e0 + j, V), cp, kp));
         const float wq = ex2_approx(fmaf(lane_block_elem<DT>(vq, j, e0 + j, V), cq, kq));
-        w[j] = fmaxf(fmaf(wp, beta, -wq), 0.f);
-    }
-    return pick_in_block<EPL>(w, e0, t, lane);
+        return fmaxf(fmaf(wp, beta, -wq), 0.f);
+    }, e0, t, lane);
 }
 
 // In one chunk: how many elements equal the row maximum m, the lowest index of one, and the largest

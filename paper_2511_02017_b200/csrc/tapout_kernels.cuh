@@ -19,29 +19,21 @@ namespace tpo {
 namespace cg = cooperative_groups;
 
 constexpr int kMaxCluster = 8;           // portable cluster size limit
+constexpr int kFinishThreads = 128;       // k_draft_finish: four rows per CTA, no register ceiling
 constexpr int kResident = 4;              // CTAs of a streaming kernel resident per SM (64 registers per thread)
-constexpr int kTodo = 32;                // rows a CTA may queue for finishing after its streaming loop
 
-struct WarpRec { float ref, k, S, T, c1, c2; int best; int pad; };
-
-// How many CTAs share one draft row, decided on the device from the number of rows actually drafted at
-// this position (the host never learns it): the smallest split whose items fill at least 90 % of a whole
-// number of waves of the persistent grid, else the best-filling one; never less than a chunk per warp.
-__device__ __forceinline__ int segments_for(const Params& p, int n_rows, int grid) {
-    if (p.nseg > 0) return p.nseg;
-    const unsigned cap = (unsigned)max(1, min(min(kMaxSeg, p.NC), max(p.NC / kWarps, 1)));
+// Into how many segments a draft row is cut, one warp per segment, decided on the device from the number
+// of rows actually drafted at this position (the host never learns it).  Many rows: about three items per
+// warp of the grid so that the ticket counter can even out slow and fast SMs, but segments of at least
+// eight chunks so that a segment's epilogue stays small beside its streaming.  Few rows: as many segments
+// as it takes to give every warp of the grid something to read, down to one chunk per segment.
+__device__ __forceinline__ int segments_for(const Params& p, int n_rows, int n_warps) {
+    const int cap = max(1, min(kMaxSeg, p.NC));
+    if (p.nseg > 0) return min(p.nseg, cap);
     if (n_rows <= 0) return 1;
-    const unsigned n = (unsigned)n_rows, G = (unsigned)grid;     // n * cap < 2^31: n_seq is bounded at create
-    unsigned best = 1;
-    float best_fill = 0.f;
-    for (unsigned k = 1; k <= cap; ++k) {
-        const unsigned items = n * k;
-        const unsigned slots = (items + G - 1) / G * G;
-        const float fill = (float)items / (float)slots;
-        if (fill >= 0.9f) return (int)k;
-        if (fill > best_fill) { best = k; best_fill = fill; }
-    }
-    return (int)best;
+    int nseg = min((3 * n_warps + n_rows - 1) / n_rows, max(p.NC / 8, 1));
+    if ((long long)n_rows * nseg < n_warps) nseg = (n_warps + n_rows - 1) / n_rows;
+    return max(1, min(nseg, cap));
 }
 
 // One warp's share of the chunks [c0, c1) of a row: chunk c0 + warp, then every kWarps-th.  Loads are not
@@ -88,31 +80,50 @@ __device__ __forceinline__ void store_segrec(SegRec* g, const SegRec& r) {
 // Finishes one row once all of its segments are reduced (one warp).  Draft position: Table 1 features,
 // x_i ~ softmax(row), the stop rule of the arm chosen for this position, bookkeeping, and the list for
 // the next position.  FEATURES (tapout_row_stats): the features only, nothing of the round's state is
-// touched.  Two dependent trips to memory: the segment records with the chunk partials, then the two
-// 2 KB chunks that hold the row maximum and the drawn token.
+// touched.  Two dependent trips to memory: the segment records with the chunk partials (and the few
+// state words the rule needs), then the two 2 KB chunks that hold the row maximum and the drawn token.
 template <int DT, bool FEATURES>
 __device__ __forceinline__ void finish_row(const Params& p, const State& st, const Scratch& sc, const StepArgs& a, int s,
-                                        int nseg, int lane) {
+                                           int nseg, int lane) {
     const char* row = reinterpret_cast<const char*>(a.logits) + (size_t)s * a.row_stride * Elem<DT>::BYTES;
     const float2* part = sc.cdf + (size_t)s * p.NC;
     const float c = a.c;
     const int pos = a.pos;
 
-    // ---- segment records and chunk partials
-    SegRec r;
-    r.ref = neg_inf(); r.S = 0.f; r.T = 0.f; r.c2 = neg_inf(); r.best = -1;
-    if (lane < nseg) r = load_segrec(sc.seg + (size_t)s * kMaxSeg + lane);
+    // ---- first trip: segment records (two per lane), chunk partials, rule state
+    SegRec r[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        r[j].ref = neg_inf(); r[j].S = 0.f; r[j].T = 0.f; r[j].c2 = neg_inf(); r[j].best = -1;
+        if (lane + 32 * j < nseg) r[j] = load_segrec(sc.seg + (size_t)s * kMaxSeg + lane + 32 * j);
+    }
     const bool in_regs = p.NC <= 32 * kRegPer;
     RegCdf cdf;
     if (in_regs) cdf.load(part, p.NC, lane);
-    const bool has_nan = __any_sync(0xffffffffu, (r.S != r.S) || (r.T != r.T) || (r.ref != r.ref));
-    const float m = warp_max_f(r.ref);
+    int arm = 0;
+    double sq_prev = 0.0, lambda = 0.0;
+    if (!FEATURES && lane == 0) {
+        arm = st.arm[(size_t)s * p.K + pos];
+        sq_prev = st.sqrtH_prev[s];
+        lambda = st.lambda[s];
+    }
+    bool has_nan = false;
+    float m = neg_inf();
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        has_nan = has_nan || (r[j].S != r[j].S) || (r[j].T != r[j].T) || (r[j].ref != r[j].ref);
+        m = fmaxf(m, r[j].ref);
+    }
+    has_nan = __any_sync(0xffffffffu, has_nan);
+    m = warp_max_f(m);
     const double mc = (double)m * (double)c;
     double Tg = 0.0;
-    if (lane < nseg && r.ref > neg_inf() && r.ref < CUDART_INF_F) {
-        const double d = (double)__fmul_rn(-r.ref, c) + mc;              // >= 0 up to rounding
-        Tg = exp2(-d) * ((double)r.T - d * (double)r.S);
-    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+        if (r[j].ref > neg_inf() && r[j].ref < CUDART_INF_F) {
+            const double d = (double)__fmul_rn(-r[j].ref, c) + mc;       // >= 0 up to rounding
+            Tg += exp2(-d) * ((double)r[j].T - d * (double)r[j].S);
+        }
     const double T2 = warp_sum_d(Tg);                                    // sum of w * t (log2 units)
     CdfTotals tot;
     double W;
@@ -120,7 +131,6 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     else { tot = cdf_totals<true>(part, p.NC, c, mc, true, lane); W = tot.W; }
     const bool valid = !has_nan && (m > neg_inf()) && (m < CUDART_INF_F) && (W > 0.0) && (W < CUDART_INF);
 
-    if (lane == 0) sc.done[s] = 0;
     if (!FEATURES && lane == 0) atomicAdd(&sc.status[1], 1ull);
     if (!valid) {
         if (lane == 0) {
@@ -137,12 +147,14 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
         return;
     }
 
-    // ---- which chunk holds the maximum (lowest such), which one the drawn token
-    const unsigned tie = __ballot_sync(0xffffffffu, lane < nseg && r.ref == m);
-    const int win = __ffs(tie) - 1;
-    const float other = warp_max_f((lane == win || lane >= nseg) ? neg_inf() : r.ref);
-    const float c2all = warp_max_f(r.c2);
-    const int best = max(__shfl_sync(0xffffffffu, r.best, win), 0);
+    // ---- which chunk holds the maximum (the lowest such), which one the drawn token
+    const unsigned tie0 = __ballot_sync(0xffffffffu, r[0].best >= 0 && r[0].ref == m);
+    const unsigned tie1 = __ballot_sync(0xffffffffu, r[1].best >= 0 && r[1].ref == m);
+    const int win = tie0 ? __ffs(tie0) - 1 : 32 + __ffs(tie1) - 1;      // segments are in token order
+    const int best = max(__shfl_sync(0xffffffffu, win < 32 ? r[0].best : r[1].best, win & 31), 0);
+    const float other = warp_max_f(fmaxf(lane == win ? neg_inf() : r[0].ref, lane + 32 == win ? neg_inf() : r[1].ref));
+    const float c2all = warp_max_f(fmaxf(r[0].c2, r[1].c2));
+    const int n_tie = __popc(tie0) + __popc(tie1);
     int chunk = 0;
     double rem = 0.0;
     float refc = 0.f;
@@ -151,29 +163,29 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
         const uint4 w = rng_words(p, seq, a.round, (uint32_t)pos, RNG_DRAFT, 0, 0);
         const double tgt = u24_to_double(w.x) * W;
         if (in_regs) {
-            chunk = cdf.locate(tgt, lane, rem, refc);
+            chunk = cdf.locate(tgt, lane, c, mc, rem, refc);
         } else {
             chunk = cdf_locate<true>(part, p.NC, c, mc, true, lane, tot, tgt, rem);
             if (chunk >= 0) refc = __ldcg(part + chunk).x;
         }
     }
+    // ---- second trip: both chunks on their way while the features are worked out
     uint4 vt[4], vx[4];
     load_lane_block<DT>(row, p.V, best, lane, vt);
     if (!FEATURES) load_lane_block<DT>(row, p.V, max(chunk, 0), lane, vx);
 
-    // ---- features (Table 1): while the two chunks are on their way
     const float inv_T = FEATURES ? a.inv_T : p.inv_Tq;
     const double lw = log(W);
     const double m_s = (double)m * (double)inv_T;
     const double lse = m_s + lw;
     const double p1 = 1.0 / W;
-    double H = lw - kLn2 * T2 / W;
+    double H = lw - kLn2 * T2 * p1;
     H = H > 0.0 ? H : 0.0;
     int cnt, first;
     float below;
     scan_top_block<DT>(vt, p.V, best, m, lane, cnt, first, below);
-    const float m2 = (__popc(tie) >= 2 || cnt >= 2) ? m : fmaxf(fmaxf(other, c2all), below);
-    const double p2 = (m2 > neg_inf()) ? exp(((double)m2 - (double)m) * (double)inv_T) / W : 0.0;
+    const float m2 = (n_tie >= 2 || cnt >= 2) ? m : fmaxf(fmaxf(other, c2all), below);
+    const double p2 = (m2 > neg_inf()) ? exp(((double)m2 - (double)m) * (double)inv_T) * p1 : 0.0;
 
     if (FEATURES) {
         if (lane == 0) {
@@ -195,8 +207,10 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
         fo[0] = (float)m_s; fo[1] = (float)lse; fo[2] = (float)p1; fo[3] = (float)p2; fo[4] = (float)H;
         fo[5] = (float)first;
         st.lse_q[(size_t)s * p.K + pos] = lse;
-        const int arm = st.arm[(size_t)s * p.K + pos];
-        bool stop = rule_stop(p, p.rule_of_arm[arm], p1, p2, H, st.sqrtH_prev[s], pos > 0, st.lambda[s]);
+        int rule = 0;                        // a select chain: indexing the parameter array would move it to local memory
+#pragma unroll
+        for (int k = 0; k < kMaxArms; ++k) rule = (k == arm) ? p.rule_of_arm[k] : rule;
+        bool stop = rule_stop(p, rule, p1, p2, H, sq_prev, pos > 0, lambda);
         st.sqrtH_prev[s] = sqrt(H);
         if (pos == p.K - 1) stop = true;
         st.n_drafted[s] = pos + 1;
@@ -222,31 +236,27 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
 // ============================================================================================
 template <int DT, bool FEATURES>
 __global__ void __launch_bounds__(kThreads, kResident)
-k_draft_step(Params p, State st, Scratch sc, StepArgs a)
+k_draft_stream(Params p, Scratch sc, StepArgs a)
 {
     constexpr int ESZ = Elem<DT>::BYTES;
-    __shared__ WarpRec wrec[2][kWarps];
-    __shared__ int todo[kTodo];              // rows whose last segment this CTA reduced: finished after the streaming
-    __shared__ int n_todo;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) n_todo = 0;
+    const int lane = threadIdx.x & 31;
+    const int gw = (int)((blockIdx.x * kThreads + threadIdx.x) >> 5);          // this warp in the grid
+    const int n_warps = (int)((gridDim.x * kThreads) >> 5);
     pdl_trigger();
     pdl_wait();
+    int* ticket = sc.count + 4;
     const int n_rows = FEATURES ? a.n_fixed : sc.count[a.slot];
     const int32_t* list = sc.list + (size_t)a.slot * p.S;
-    if (!FEATURES) {
-        // the list two positions ahead is free again: nobody reads or appends to it during this launch
-        if (blockIdx.x == 0 && tid == 0) sc.count[(a.slot + 2) % 3] = 0;
-        // sequences that stopped at an earlier position draft nothing
-        for (int s = blockIdx.x * kThreads + tid; s < p.S; s += gridDim.x * kThreads)
-            if (sc.next_pos[s] < a.pos) { a.out_token[(size_t)s * a.tok_stride] = -1; a.out_continue[s] = 0; }
-    }
-    const int nseg = segments_for(p, n_rows, (int)gridDim.x);
+    const int nseg = segments_for(p, n_rows, n_warps);
     const int total = n_rows * nseg;
     const float c = a.c;
 
-    int it = 0;
-    for (int item = blockIdx.x; item < total; item += gridDim.x, ++it) {
+    // Work item = (row, segment), one warp each: the first n_warps items by position in the grid, the
+    // rest by ticket.  No warp ever waits for another one; the results are combined by k_draft_finish.
+    int item = gw;
+    while (item < total) {
+        int nxt = 0;
+        if (lane == 0) nxt = atomicAdd(ticket, 1);       // asked for now, needed only after this item
         const int ai = item / nseg, g = item - ai * nseg;
         const int s = FEATURES ? ai : list[ai];
         const char* row = reinterpret_cast<const char*>(a.logits) + (size_t)s * a.row_stride * ESZ;
@@ -256,56 +266,49 @@ k_draft_step(Params p, State st, Scratch sc, StepArgs a)
 
         WarpAcc acc;
         acc.init();
-        stream_chunks<DT, true, true>(acc, row, p.V, c0, c1, warp, lane, c,
-                                      [&](int ch, float ref, float tot) { part[ch] = make_float2(ref, tot); });
+        for (int ch = c0; ch < c1; ++ch) {
+            uint4 v[kVecPerLane];
+            load_chunk<DT>(row, p.V, ch, lane, v);
+            const float tot = fold_chunk<DT, true, true>(acc, v, ch, c);
+            if (lane == 0) part[ch] = make_float2(acc.ref, tot);
+        }
         const float Sw = warp_sum_f(acc.S), Tw = warp_sum_f(acc.T);
-        const int buf = it & 1;
         if (lane == 0) {
-            WarpRec r;
-            r.ref = acc.ref; r.k = acc.k; r.S = Sw; r.T = Tw; r.c1 = acc.c1; r.c2 = acc.c2; r.best = acc.best; r.pad = 0;
-            wrec[buf][warp] = r;
+            SegRec o;
+            o.ref = acc.ref; o.S = Sw; o.T = Tw; o.c2 = acc.c2; o.best = acc.best;
+            o.pad0 = o.pad1 = o.pad2 = 0;
+            store_segrec(sc.seg + (size_t)s * kMaxSeg + g, o);
         }
-        __syncthreads();                     // also orders every warp's chunk partials before the fence below
-        if (warp == (it & (kWarps - 1))) {   // the merging warp rotates; the others run ahead into the next item
-            // lane w merges warp w's record: common reference = the largest, sums rescaled to it
-            WarpRec r;
-            r.ref = neg_inf(); r.k = 0.f; r.S = 0.f; r.T = 0.f; r.c1 = neg_inf(); r.c2 = neg_inf(); r.best = -1;
-            if (lane < kWarps) r = wrec[buf][lane];
-            const bool live = r.ref != neg_inf();                 // a NaN reference counts as live and poisons S
-            const float ref = warp_max_f(r.ref);
-            const float kref = __fmul_rn(-ref, c);
-            const float dd = live ? kref - r.k : 0.f;             // <= 0
-            const float f = live ? ex2_approx(dd) : 0.f;
-            const float Sg = warp_sum_f(live ? f * r.S : 0.f);
-            const float Tg = warp_sum_f(live ? f * fmaf(dd, r.S, r.T) : 0.f);
-            // two largest chunk maxima of the segment (with multiplicity); lowest chunk holding the largest
-            const unsigned tie = __ballot_sync(0xffffffffu, r.best >= 0 && r.c1 == ref);
-            const int win = tie ? __ffs(tie) - 1 : 0;
-            const float other = warp_max_f((lane == win) ? neg_inf() : r.c1);
-            const float c2all = warp_max_f(r.c2);
-            const float C2 = (__popc(tie) >= 2) ? ref : fmaxf(other, c2all);
-            const int best = __reduce_min_sync(0xffffffffu, (tie >> lane) & 1u ? r.best : 0x7fffffff);
-            int last = 0;
-            if (lane == 0) {
-                SegRec o;
-                o.ref = ref; o.S = Sg; o.T = Tg; o.c2 = C2; o.best = (best == 0x7fffffff) ? -1 : best;
-                o.pad0 = o.pad1 = o.pad2 = 0;
-                store_segrec(sc.seg + (size_t)s * kMaxSeg + g, o);
-                __threadfence();             // the segment (record and chunk partials) before it is counted
-                last = atomicAdd(&sc.done[s], 1) == nseg - 1;
-                if (last && n_todo < kTodo) { todo[n_todo] = s; n_todo = n_todo + 1; last = 0; }
-            }
-            last = __shfl_sync(0xffffffffu, last, 0);
-            if (last) {                      // queue full: finish at once
-                __threadfence();
-                finish_row<DT, FEATURES>(p, st, sc, a, s, nseg, lane);
-            }
-        }
+        item = __shfl_sync(0xffffffffu, nxt, 0) + n_warps;
     }
-    __syncthreads();
-    // the rows this CTA completed, one warp each; their other segments were published before they were counted
-    if (n_todo > 0) __threadfence();
-    for (int j = warp; j < n_todo; j += kWarps) finish_row<DT, FEATURES>(p, st, sc, a, todo[j], nseg, lane);
+}
+
+// Second kernel of a draft position: one warp per row that was streamed (finish_row), the outputs of
+// the sequences that had stopped before, and the hand-over of the lists to the next position.
+// n_warps_stream: warps of the k_draft_stream grid that cut the rows (the split must be recomputed alike).
+template <int DT, bool FEATURES>
+__global__ void __launch_bounds__(kFinishThreads)
+k_draft_finish(Params p, State st, Scratch sc, StepArgs a, int n_warps_stream)
+{
+    const int lane = threadIdx.x & 31;
+    const int gw = (int)((blockIdx.x * kFinishThreads + threadIdx.x) >> 5);
+    const int n_warps = (int)((gridDim.x * kFinishThreads) >> 5);
+    pdl_trigger();
+    pdl_wait();
+    const int n_rows = FEATURES ? a.n_fixed : sc.count[a.slot];
+    if (gw == 0 && lane == 0) {
+        sc.count[4] = 0;                                 // the work ticket of the next streaming kernel
+        if (!FEATURES) sc.count[(a.slot + 2) % 3] = 0;   // the list two positions ahead is free again
+    }
+    if (!FEATURES) {
+        // sequences that stopped at an earlier position draft nothing
+        for (int s = blockIdx.x * kFinishThreads + threadIdx.x; s < p.S; s += gridDim.x * kFinishThreads)
+            if (sc.next_pos[s] < a.pos) { a.out_token[(size_t)s * a.tok_stride] = -1; a.out_continue[s] = 0; }
+    }
+    const int nseg = segments_for(p, n_rows, n_warps_stream);
+    const int32_t* list = sc.list + (size_t)a.slot * p.S;
+    for (int ai = gw; ai < n_rows; ai += n_warps)
+        finish_row<DT, FEATURES>(p, st, sc, a, FEATURES ? ai : list[ai], nseg, lane);
 }
 
 // ============================================================================================
@@ -610,7 +613,7 @@ __device__ __forceinline__ void begin_round(const Params& p, const State& st, co
     if (lane == 0) {
         st.active[s] = 1; st.n_drafted[s] = 0; st.sqrtH_prev[s] = 0.0;
         sc.list[s] = s; sc.next_pos[s] = 0; sc.done[s] = 0;
-        if (s == 0) { sc.count[0] = p.S; sc.count[1] = 0; sc.count[2] = 0; sc.count[3] = 0; }
+        if (s == 0) { sc.count[0] = p.S; sc.count[1] = 0; sc.count[2] = 0; sc.count[3] = 0; sc.count[4] = 0; }
     }
 }
 

@@ -394,3 +394,32 @@ def test_seq_offset_shards_reproduce_the_full_batch():
             assert torch.equal(f[j], torch.cat([parts[0][j], parts[1][j]]))
     for hnd in [full] + halves:
         hnd.destroy()
+
+
+def test_round_call_matches_separate_calls():
+    """tapout_round enqueues the same kernels as k_max draft steps + verify + update."""
+    w = si.Workload("rnd", 7, 4104, "bf16", 5, 1, 5, "ts", "token", seed=61)
+    from tests.lockstep import make_device
+    a, b = make_device(w), make_device(w)
+    S, K = w.n_seq, w.k_max
+    tok = torch.empty(S, dtype=torch.int32, device=DEV)
+    cont = torch.empty(S, dtype=torch.uint8, device=DEV)
+    acc = torch.empty(S, dtype=torch.int32, device=DEV)
+    nxt = torch.empty(S, dtype=torch.int32, device=DEV)
+    toks_b = torch.empty((S, K), dtype=torch.int32, device=DEV)
+    cont_b = torch.empty(S, dtype=torch.uint8, device=DEV)
+    acc_b = torch.empty(S, dtype=torch.int32, device=DEV)
+    nxt_b = torch.empty(S, dtype=torch.int32, device=DEV)
+    for rnd in range(8):
+        d, t = peaked_logits(w, rnd, DEV)
+        toks = torch.full((S, K), -1, dtype=torch.int32, device=DEV)
+        for i in range(K):
+            a.draft_step(d[:, i, :], tok, cont)
+            toks[:, i] = tok
+        a.verify(d, t, toks, acc, nxt)
+        a.update()
+        b.round(d, t, toks_b, cont_b, acc_b, nxt_b)
+        assert torch.equal(toks, toks_b) and torch.equal(acc, acc_b) and torch.equal(nxt, nxt_b)
+    assert np.array_equal(a.get_state()["_blob"], b.get_state()["_blob"])
+    a.destroy()
+    b.destroy()
