@@ -397,14 +397,19 @@ constexpr int kRegPer = 8;
 // part.y * 2^-(k_ch + mc) like chunk_contrib, but with the power of two taken apart: integer part by
 // exponent arithmetic, fraction by the fp32 exponential unit (relative error about 2e-7, the accuracy of
 // the partial sums themselves).
-__device__ __forceinline__ double scaled_contrib(float2 p, float c, double mc) {
-    if (!(p.y > 0.f)) return (p.y != p.y) ? (double)p.y : 0.0;
-    const double d = (double)__fmul_rn(-p.x, c) + mc;                     // >= 0 up to rounding
+// 2^-d for d >= 0 (up to rounding) with the power of two taken apart: integer part by exponent arithmetic,
+// fraction by the fp32 exponential unit.  Relative error about 2e-7.
+__device__ __forceinline__ double pow2_neg(double d) {
     const double dn = floor(d);
     if (dn > 1000.0) return 0.0;
     const int n = (int)dn;
     const float fr = (float)(d - dn);
-    return (double)p.y * (double)ex2_approx(-fr) * __hiloint2double((1023 - n) << 20, 0);
+    return (double)ex2_approx(-fr) * __hiloint2double((1023 - n) << 20, 0);
+}
+
+__device__ __forceinline__ double scaled_contrib(float2 p, float c, double mc) {
+    if (!(p.y > 0.f)) return (p.y != p.y) ? (double)p.y : 0.0;
+    return (double)p.y * pow2_neg((double)__fmul_rn(-p.x, c) + mc);         // the exponent is >= 0 up to rounding
 }
 
 struct RegCdf {
@@ -495,14 +500,15 @@ __device__ __forceinline__ float lane_block_elem(const uint4 (&v)[4], int k, int
 // Token inside one chunk.  Lane l owns the EPL consecutive tokens starting at first_token (its own);
 // weight(k) gives the weight (>= 0) of its k-th token exactly as the streaming pass formed it, t is the
 // target inside the chunk in the same units.  First token whose running sum exceeds t; if rounding
-// leaves none, the last token with positive weight.  Sums run in double so that the order of additions
-// cannot matter.  The weights are formed twice (once for the lane totals, once for the walk inside the
+// leaves none, the last token with positive weight.  Across lanes the sums run in double; inside a lane
+// (32 or 16 tokens) in fp32, whose error is far below that of the chunk partials.  The weights are formed twice (once for the lane totals, once for the walk inside the
 // chosen lane) instead of being kept in an array of registers.
 template <int EPL, typename Weight>
 __device__ __forceinline__ int pick_in_block(Weight weight, int first_token, double t, int lane) {
-    double sum = 0.0;
+    float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-    for (int k = 0; k < EPL; ++k) sum += (double)weight(k);
+    for (int k = 0; k < EPL; k += 2) { s0 += weight(k); s1 += weight(k + 1); }
+    const double sum = (double)s0 + (double)s1;
     const double incl = warp_incl_scan_d(sum, lane);
     const unsigned over = __ballot_sync(0xffffffffu, incl > t);
     const unsigned pos = __ballot_sync(0xffffffffu, sum > 0.0);
@@ -510,13 +516,13 @@ __device__ __forceinline__ int pick_in_block(Weight weight, int first_token, dou
     if (over) L = __ffs(over) - 1;
     else if (pos) L = 31 - __clz(pos);
     else return -1;
-    const double tl = t - (incl - sum);
-    double run = 0.0;
+    const float tl = (float)(t - (incl - sum));          // inside one lane's 64 bytes fp32 carries the walk
+    float run = 0.f;
     int pick = -1, last_pos = -1;
 #pragma unroll
     for (int k = 0; k < EPL; ++k) {
-        const double x = (double)weight(k);
-        if (x > 0.0) last_pos = k;
+        const float x = weight(k);
+        if (x > 0.f) last_pos = k;
         run += x;
         if (pick < 0 && run > tl) pick = k;
     }

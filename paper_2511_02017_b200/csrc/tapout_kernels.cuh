@@ -25,13 +25,13 @@ constexpr int kResident = 4;              // CTAs of a streaming kernel resident
 // Into how many segments a draft row is cut, one warp per segment, decided on the device from the number
 // of rows actually drafted at this position (the host never learns it).  Many rows: about three items per
 // warp of the grid so that the ticket counter can even out slow and fast SMs, but segments of at least
-// eight chunks so that a segment's epilogue stays small beside its streaming.  Few rows: as many segments
+// six chunks so that a segment's epilogue stays small beside its streaming.  Few rows: as many segments
 // as it takes to give every warp of the grid something to read, down to one chunk per segment.
 __device__ __forceinline__ int segments_for(const Params& p, int n_rows, int n_warps) {
     const int cap = max(1, min(kMaxSeg, p.NC));
     if (p.nseg > 0) return min(p.nseg, cap);
     if (n_rows <= 0) return 1;
-    int nseg = min((3 * n_warps + n_rows - 1) / n_rows, max(p.NC / 8, 1));
+    int nseg = min((3 * n_warps + n_rows - 1) / n_rows, max(p.NC / 6, 1));
     if ((long long)n_rows * nseg < n_warps) nseg = (n_warps + n_rows - 1) / n_rows;
     return max(1, min(nseg, cap));
 }
@@ -84,19 +84,20 @@ __device__ __forceinline__ void store_segrec(SegRec* g, const SegRec& r) {
 // state words the rule needs), then the two 2 KB chunks that hold the row maximum and the drawn token.
 template <int DT, bool FEATURES>
 __device__ __forceinline__ void finish_row(const Params& p, const State& st, const Scratch& sc, const StepArgs& a, int s,
-                                           int nseg, int lane) {
+                                           int n_warps_stream, int lane) {
     const char* row = reinterpret_cast<const char*>(a.logits) + (size_t)s * a.row_stride * Elem<DT>::BYTES;
     const float2* part = sc.cdf + (size_t)s * p.NC;
     const float c = a.c;
     const int pos = a.pos;
 
-    // ---- first trip: segment records (two per lane), chunk partials, rule state
+    // ---- first trip, everything at once: is the sequence drafting at this position, how many rows are
+    // (the split follows from it), all 64 segment-record slots (two per lane; those beyond the split are
+    // stale and masked below), chunk partials, rule state.  Nothing here waits for anything else.
+    const int np = FEATURES ? pos : __ldcg(sc.next_pos + s);
+    const int n_rows = FEATURES ? a.n_fixed : __ldcg(sc.count + a.slot);
     SegRec r[2];
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-        r[j].ref = neg_inf(); r[j].S = 0.f; r[j].T = 0.f; r[j].c2 = neg_inf(); r[j].best = -1;
-        if (lane + 32 * j < nseg) r[j] = load_segrec(sc.seg + (size_t)s * kMaxSeg + lane + 32 * j);
-    }
+    for (int j = 0; j < 2; ++j) r[j] = load_segrec(sc.seg + (size_t)s * kMaxSeg + lane + 32 * j);
     const bool in_regs = p.NC <= 32 * kRegPer;
     RegCdf cdf;
     if (in_regs) cdf.load(part, p.NC, lane);
@@ -107,6 +108,18 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
         sq_prev = st.sqrtH_prev[s];
         lambda = st.lambda[s];
     }
+    // the uniform of the token draw does not depend on anything loaded: worked out while the loads fly
+    double u_draw = 0.0;
+    if (!FEATURES) u_draw = u24_to_double(rng_words(p, p.seq_offset + (uint32_t)s, a.round, (uint32_t)pos, RNG_DRAFT, 0, 0).x);
+    if (np != pos) {
+        // stopped at an earlier position: drafts nothing
+        if (lane == 0 && np < pos) { a.out_token[(size_t)s * a.tok_stride] = -1; a.out_continue[s] = 0; }
+        return;
+    }
+    const int nseg = segments_for(p, n_rows, n_warps_stream);
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+        if (lane + 32 * j >= nseg) { r[j].ref = neg_inf(); r[j].S = 0.f; r[j].T = 0.f; r[j].c2 = neg_inf(); r[j].best = -1; }
     bool has_nan = false;
     float m = neg_inf();
 #pragma unroll
@@ -122,7 +135,7 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     for (int j = 0; j < 2; ++j)
         if (r[j].ref > neg_inf() && r[j].ref < CUDART_INF_F) {
             const double d = (double)__fmul_rn(-r[j].ref, c) + mc;       // >= 0 up to rounding
-            Tg += exp2(-d) * ((double)r[j].T - d * (double)r[j].S);
+            Tg += pow2_neg(d) * ((double)r[j].T - d * (double)r[j].S);
         }
     const double T2 = warp_sum_d(Tg);                                    // sum of w * t (log2 units)
     CdfTotals tot;
@@ -159,9 +172,7 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     double rem = 0.0;
     float refc = 0.f;
     if (!FEATURES) {
-        const uint32_t seq = p.seq_offset + (uint32_t)s;
-        const uint4 w = rng_words(p, seq, a.round, (uint32_t)pos, RNG_DRAFT, 0, 0);
-        const double tgt = u24_to_double(w.x) * W;
+        const double tgt = u_draw * W;
         if (in_regs) {
             chunk = cdf.locate(tgt, lane, c, mc, rem, refc);
         } else {
@@ -185,7 +196,11 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     float below;
     scan_top_block<DT>(vt, p.V, best, m, lane, cnt, first, below);
     const float m2 = (n_tie >= 2 || cnt >= 2) ? m : fmaxf(fmaxf(other, c2all), below);
-    const double p2 = (m2 > neg_inf()) ? exp(((double)m2 - (double)m) * (double)inv_T) * p1 : 0.0;
+    // two exponentials from one call: lane 1 works out the scale of the token draw, the others p2
+    const float kch = __fmul_rn(-refc, c);
+    const double ex = exp(lane == 1 ? kLn2 * ((double)kch + mc) : ((double)m2 - (double)m) * (double)inv_T);
+    const double p2 = (m2 > neg_inf()) ? ex * p1 : 0.0;
+    const double draw_scale = __shfl_sync(0xffffffffu, ex, 1);            // 2^(kch + mc)
 
     if (FEATURES) {
         if (lane == 0) {
@@ -198,10 +213,7 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
 
     // ---- x_i ~ softmax(row) inside the chunk, from the weights the streaming pass summed
     int tok = -1;
-    if (chunk >= 0) {
-        const float kch = __fmul_rn(-refc, c);
-        tok = pick_softmax_block<DT>(vx, p.V, chunk, c, kch, rem * exp2((double)kch + mc), lane);
-    }
+    if (chunk >= 0) tok = pick_softmax_block<DT>(vx, p.V, chunk, c, kch, rem * draw_scale, lane);
     if (lane == 0) {
         float* fo = st.feat + ((size_t)s * p.K + pos) * kFeat;
         fo[0] = (float)m_s; fo[1] = (float)lse; fo[2] = (float)p1; fo[3] = (float)p2; fo[4] = (float)H;
@@ -283,9 +295,10 @@ k_draft_stream(Params p, Scratch sc, StepArgs a)
     }
 }
 
-// Second kernel of a draft position: one warp per row that was streamed (finish_row), the outputs of
-// the sequences that had stopped before, and the hand-over of the lists to the next position.
-// n_warps_stream: warps of the k_draft_stream grid that cut the rows (the split must be recomputed alike).
+// Second kernel of a draft position: one warp per sequence (finish_row; a sequence that is not drafting
+// at this position only gets its "nothing drafted" outputs), and the hand-over of the lists to the next
+// position.  n_warps_stream: warps of the k_draft_stream grid that cut the rows (the split is recomputed
+// alike).  FEATURES: rows 0 .. n_fixed-1.
 template <int DT, bool FEATURES>
 __global__ void __launch_bounds__(kFinishThreads)
 k_draft_finish(Params p, State st, Scratch sc, StepArgs a, int n_warps_stream)
@@ -295,20 +308,12 @@ k_draft_finish(Params p, State st, Scratch sc, StepArgs a, int n_warps_stream)
     const int n_warps = (int)((gridDim.x * kFinishThreads) >> 5);
     pdl_trigger();
     pdl_wait();
-    const int n_rows = FEATURES ? a.n_fixed : sc.count[a.slot];
     if (gw == 0 && lane == 0) {
         sc.count[4] = 0;                                 // the work ticket of the next streaming kernel
         if (!FEATURES) sc.count[(a.slot + 2) % 3] = 0;   // the list two positions ahead is free again
     }
-    if (!FEATURES) {
-        // sequences that stopped at an earlier position draft nothing
-        for (int s = blockIdx.x * kFinishThreads + threadIdx.x; s < p.S; s += gridDim.x * kFinishThreads)
-            if (sc.next_pos[s] < a.pos) { a.out_token[(size_t)s * a.tok_stride] = -1; a.out_continue[s] = 0; }
-    }
-    const int nseg = segments_for(p, n_rows, n_warps_stream);
-    const int32_t* list = sc.list + (size_t)a.slot * p.S;
-    for (int ai = gw; ai < n_rows; ai += n_warps)
-        finish_row<DT, FEATURES>(p, st, sc, a, FEATURES ? ai : list[ai], nseg, lane);
+    const int n = FEATURES ? a.n_fixed : p.S;
+    for (int s = gw; s < n; s += n_warps) finish_row<DT, FEATURES>(p, st, sc, a, s, n_warps_stream, lane);
 }
 
 // ============================================================================================
