@@ -39,6 +39,30 @@ def measured_peaks():
     return 6650.0, "fallback (earlier measurement on this pool)"
 
 
+def kernel_source_digest():
+    """Digest of the CUDA sources: DRAM counters taken from an older build of the kernels are not reported."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2511_02017_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        h.update(open(os.path.join(csrc, name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def measured_traffic(kernel, alg_bytes_per_launch):
+    """DRAM bytes per launch from the committed ncu capture (profiles/dram_traffic.json: DRAM bytes moved per
+    algorithmic byte on a smaller case of the same kernels), scaled to this launch; None if the kernels have
+    changed since the capture."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        rec = json.load(open(path))
+        if rec.get("source_digest") != kernel_source_digest() or kernel not in rec["dram_bytes_per_alg_byte"]:
+            return None
+        return rec["dram_bytes_per_alg_byte"][kernel] * alg_bytes_per_launch
+    except Exception:
+        return None
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
 
@@ -231,11 +255,13 @@ def bench_ours(args):
         ms_k, n_k = prof[k]
         return {"launches": n_k, "ms_total": ms_k, "alg_bytes": rows_k * row_bytes,
                 "gbs": rows_k * row_bytes / (ms_k * 1e-3) / 1e9 if ms_k > 0 else None}
-    kernels = {"k_draft_step": kinfo(0, d_rows), "k_verify_walk": kinfo(1, v_rows), "k_update": kinfo(2, 0)}
+    kernels = {"k_draft_stream+k_draft_finish": kinfo(0, d_rows), "k_verify_walk": kinfo(1, v_rows),
+               "k_update": kinfo(2, 0)}
     dom = max(kernels, key=lambda k: kernels[k]["ms_total"])
     achieved = kernels[dom]["gbs"] or 0.0
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+                "frac": achieved / peak, "peak_source": peak_src,
+                "traffic": measured_traffic(dom, kernels[dom]["alg_bytes"] / max(1, kernels[dom]["launches"])),
                 "alg_bytes_per_launch": kernels[dom]["alg_bytes"] / max(1, kernels[dom]["launches"]),
                 "avg_launch_ms": kernels[dom]["ms_total"] / max(1, kernels[dom]["launches"]),
                 "whole_step_gbs": rows * row_bytes / (ms * 1e-3) / 1e9,
@@ -278,6 +304,7 @@ def bench_ours(args):
                "sample": "%d of %d sequences, %d round(s) of this workload's logits, %d rows in %.1f s" %
                          (n_s, S, args.cpu_sample_rounds, rows_o, dt_o)}
 
+    life = dev.get_status()
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -291,6 +318,7 @@ def bench_ours(args):
                        "sharding": "independent sequences per GPU, no collective" if world > 1 else "single GPU"},
             "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "roofline": roofline, "kernels": kernels,
             "rows": {"draft": rows_d, "target": rows_t, "residual": rows_r},
+            "rows_lifetime": {"draft": life["rows_draft"], "target": life["rows_target"], "residual": life["rows_residual"]},
             "hbm_gbs": rows * row_bytes / (ms * 1e-3) / 1e9,
             "cpu_baseline": cpu,
         }
