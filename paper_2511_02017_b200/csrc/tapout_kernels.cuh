@@ -255,9 +255,14 @@ k_draft_stream(Params p, Scratch sc, StepArgs a)
     const int gw = (int)((blockIdx.x * kThreads + threadIdx.x) >> 5);          // this warp in the grid
     const int n_warps = (int)((gridDim.x * kThreads) >> 5);
     pdl_trigger();
-    pdl_wait();
+    // Position 0 reads nothing its predecessors in the stream write (every sequence drafts, in index order;
+    // the ticket was zeroed by the last finish kernel), so it starts at once and overlaps the tail of the
+    // previous round's verification and its update; it waits for them only before it exits, which is what
+    // the finish kernel behind it relies on.
+    const bool first = !FEATURES && a.pos == 0;
+    if (!first) pdl_wait();
     int* ticket = sc.count + 4;
-    const int n_rows = FEATURES ? a.n_fixed : sc.count[a.slot];
+    const int n_rows = FEATURES ? a.n_fixed : first ? p.S : sc.count[a.slot];
     const int32_t* list = sc.list + (size_t)a.slot * p.S;
     const int nseg = segments_for(p, n_rows, n_warps);
     const int total = n_rows * nseg;
@@ -270,7 +275,7 @@ k_draft_stream(Params p, Scratch sc, StepArgs a)
         int nxt = 0;
         if (lane == 0) nxt = atomicAdd(ticket, 1);       // asked for now, needed only after this item
         const int ai = item / nseg, g = item - ai * nseg;
-        const int s = FEATURES ? ai : list[ai];
+        const int s = (FEATURES || first) ? ai : list[ai];
         const char* row = reinterpret_cast<const char*>(a.logits) + (size_t)s * a.row_stride * ESZ;
         const int c0 = (int)(((long long)g * p.NC) / nseg);
         const int c1 = (int)(((long long)(g + 1) * p.NC) / nseg);
@@ -293,6 +298,7 @@ k_draft_stream(Params p, Scratch sc, StepArgs a)
         }
         item = __shfl_sync(0xffffffffu, nxt, 0) + n_warps;
     }
+    if (first) pdl_wait();
 }
 
 // Second kernel of a draft position: one warp per sequence (finish_row; a sequence that is not drafting
@@ -618,7 +624,7 @@ __device__ __forceinline__ void begin_round(const Params& p, const State& st, co
     if (lane == 0) {
         st.active[s] = 1; st.n_drafted[s] = 0; st.sqrtH_prev[s] = 0.0;
         sc.list[s] = s; sc.next_pos[s] = 0; sc.done[s] = 0;
-        if (s == 0) { sc.count[0] = p.S; sc.count[1] = 0; sc.count[2] = 0; sc.count[3] = 0; sc.count[4] = 0; }
+        if (s == 0) { sc.count[0] = p.S; sc.count[1] = 0; sc.count[2] = 0; sc.count[3] = 0; }
     }
 }
 
