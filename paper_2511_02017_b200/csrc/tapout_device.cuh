@@ -398,22 +398,27 @@ constexpr int kRegPer = 8;
 // exponent arithmetic, fraction by the fp32 exponential unit (relative error about 2e-7, the accuracy of
 // the partial sums themselves).
 // 2^-d for d >= 0 (up to rounding) with the power of two taken apart: integer part by exponent arithmetic,
-// fraction by the fp32 exponential unit.  Relative error about 2e-7.
-__device__ __forceinline__ double pow2_neg(double d) {
-    const double dn = floor(d);
-    if (dn > 1000.0) return 0.0;
-    const int n = (int)dn;
-    const float fr = (float)(d - dn);
-    return (double)ex2_approx(-fr) * __hiloint2double((1023 - n) << 20, 0);
+// fraction by the fp32 exponential unit.  d is rounded to fp32 first (relative error of the result about
+// 2^-24 * d from that, 2e-7 from the unit; partial sums far below the maximum are the only ones with a large d).
+// Straight-line code: no branch, so that several of these overlap.
+__device__ __forceinline__ float pow2_neg_f(double d) {
+    const float df = fminf(fmaxf((float)d, -1.f), 125.f);                // NaN -> -1, harmless: see scaled_contrib
+    const float dn = floorf(df);
+    const float w = ex2_approx(dn - df);                                  // 2^-(fraction)
+    return w * __int_as_float((127 - (int)dn) << 23);                     // times 2^-dn, exact
 }
+__device__ __forceinline__ double pow2_neg(double d) { return (double)pow2_neg_f(d); }
 
+// part.y * 2^-(k_ch + mc) like chunk_contrib.  Partials that are zero, negative (never written) or carry an
+// infinite reference give exactly 0; a NaN sum stays NaN.
 __device__ __forceinline__ double scaled_contrib(float2 p, float c, double mc) {
-    if (!(p.y > 0.f)) return (p.y != p.y) ? (double)p.y : 0.0;
-    return (double)p.y * pow2_neg((double)__fmul_rn(-p.x, c) + mc);         // the exponent is >= 0 up to rounding
+    const float v = pow2_neg_f((double)__fmul_rn(-p.x, c) + mc);
+    return (p.y > 0.f) ? (double)(p.y * v) : ((p.y != p.y) ? (double)p.y : 0.0);
 }
 
 struct RegCdf {
     float2 part[kRegPer];      // this lane's chunks: lane * per .. lane * per + per - 1
+    double con[kRegPer];       // their contributions to the row total, relative to the row maximum
     double lane_sum, incl, W;
     int per, NC;
 
@@ -431,14 +436,13 @@ struct RegCdf {
     __device__ __forceinline__ void scale(float c, double mc, int lane) {
         double ls = 0.0;
 #pragma unroll
-        for (int j = 0; j < kRegPer; ++j) ls += scaled_contrib(part[j], c, mc);
+        for (int j = 0; j < kRegPer; ++j) { con[j] = scaled_contrib(part[j], c, mc); ls += con[j]; }
         lane_sum = ls;
         incl = warp_incl_scan_d(ls, lane);
         W = __shfl_sync(0xffffffffu, incl, 31);
     }
     // Chunk in which the running sum first exceeds tgt (if rounding leaves none, the last chunk with a
-    // positive contribution), tgt minus the sum before it, and the chunk's reference logit.  The
-    // contributions are formed again rather than kept: registers are scarcer than arithmetic here.
+    // positive contribution), tgt minus the sum before it, and the chunk's reference logit.
     __device__ __forceinline__ int locate(double tgt, int lane, float c, double mc, double& rem, float& ref) const {
         const unsigned over = __ballot_sync(0xffffffffu, incl > tgt);
         const unsigned pos = __ballot_sync(0xffffffffu, lane_sum > 0.0);
@@ -453,7 +457,7 @@ struct RegCdf {
         float r_pick = 0.f, r_last = 0.f;
 #pragma unroll
         for (int j = 0; j < kRegPer; ++j) {
-            const double x = scaled_contrib(part[j], c, mc);
+            const double x = con[j];
             if (x > 0.0) { last_pos = j; before_last = run; r_last = part[j].x; }
             if (pick < 0 && run + x > tgt) { pick = j; before = run; r_pick = part[j].x; }
             run += x;

@@ -211,9 +211,7 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
         return;
     }
 
-    // ---- x_i ~ softmax(row) inside the chunk, from the weights the streaming pass summed
-    int tok = -1;
-    if (chunk >= 0) tok = pick_softmax_block<DT>(vx, p.V, chunk, c, kch, rem * draw_scale, lane);
+    // ---- stop rule and hand-over first (their atomics fly while the token is picked), then the token
     if (lane == 0) {
         float* fo = st.feat + ((size_t)s * p.K + pos) * kFeat;
         fo[0] = (float)m_s; fo[1] = (float)lse; fo[2] = (float)p1; fo[3] = (float)p2; fo[4] = (float)H;
@@ -227,7 +225,6 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
         if (pos == p.K - 1) stop = true;
         st.n_drafted[s] = pos + 1;
         st.active[s] = stop ? 0 : 1;
-        a.out_token[(size_t)s * a.tok_stride] = tok;
         a.out_continue[s] = stop ? 0 : 1;
         if (stop) {
             sc.stopped[atomicAdd(&sc.count[3], 1)] = s;
@@ -237,6 +234,10 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
             sc.list[(size_t)nslot * p.S + atomicAdd(&sc.count[nslot], 1)] = s;
         }
     }
+    // x_i ~ softmax(row) inside the chunk, from the weights the streaming pass summed
+    int tok = -1;
+    if (chunk >= 0) tok = pick_softmax_block<DT>(vx, p.V, chunk, c, kch, rem * draw_scale, lane);
+    if (lane == 0) a.out_token[(size_t)s * a.tok_stride] = tok;
 }
 
 // ============================================================================================
