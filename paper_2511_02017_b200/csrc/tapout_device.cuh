@@ -333,6 +333,18 @@ __device__ __forceinline__ float fold_chunk(WarpAcc& acc, const uint4 (&v)[kVecP
     return WANT_PART ? warp_sum_f(sc) : 0.f;
 }
 
+// 2^-d for d >= 0 (up to rounding) with the power of two taken apart: integer part by exponent arithmetic,
+// fraction by the fp32 exponential unit.  d is rounded to fp32 first (relative error of the result about
+// 2^-24 * d from that, 2e-7 from the unit; partial sums far below the maximum are the only ones with a large d).
+// Straight-line code: no branch, so that several of these overlap.
+__device__ __forceinline__ float pow2_neg_f(double d) {
+    const float df = fminf(fmaxf((float)d, -1.f), 125.f);                // NaN -> -1, harmless: see scaled_contrib
+    const float dn = floorf(df);
+    const float w = ex2_approx(dn - df);                                  // 2^-(fraction)
+    return w * __int_as_float((127 - (int)dn) << 23);                     // times 2^-dn, exact
+}
+__device__ __forceinline__ double pow2_neg(double d) { return (double)pow2_neg_f(d); }
+
 // ------------------------------------------------------------------ CDF search over chunk partials
 // contribution of chunk ch to the row total, relative to the row maximum m (mc = m*c in double):
 //   scaled  : part.y * 2^-(k_ch + mc), k_ch = fl(-part.x * c) exactly as the streaming pass used it
@@ -344,8 +356,7 @@ __device__ __forceinline__ double chunk_contrib(const float2* part, int ch, floa
     const float2 p = GLOBAL ? __ldcg(part + ch) : part[ch];
     if (!scaled) return (double)p.y;
     if (!(p.y > 0.f)) return (p.y != p.y) ? (double)p.y : 0.0;
-    const double k = (double)__fmul_rn(-p.x, c);
-    return (double)p.y * exp2(-(k + mc));
+    return (double)p.y * pow2_neg((double)__fmul_rn(-p.x, c) + mc);
 }
 
 struct CdfTotals { double lane_sum, incl, W; };
@@ -397,18 +408,6 @@ constexpr int kRegPer = 8;
 // part.y * 2^-(k_ch + mc) like chunk_contrib, but with the power of two taken apart: integer part by
 // exponent arithmetic, fraction by the fp32 exponential unit (relative error about 2e-7, the accuracy of
 // the partial sums themselves).
-// 2^-d for d >= 0 (up to rounding) with the power of two taken apart: integer part by exponent arithmetic,
-// fraction by the fp32 exponential unit.  d is rounded to fp32 first (relative error of the result about
-// 2^-24 * d from that, 2e-7 from the unit; partial sums far below the maximum are the only ones with a large d).
-// Straight-line code: no branch, so that several of these overlap.
-__device__ __forceinline__ float pow2_neg_f(double d) {
-    const float df = fminf(fmaxf((float)d, -1.f), 125.f);                // NaN -> -1, harmless: see scaled_contrib
-    const float dn = floorf(df);
-    const float w = ex2_approx(dn - df);                                  // 2^-(fraction)
-    return w * __int_as_float((127 - (int)dn) << 23);                     // times 2^-dn, exact
-}
-__device__ __forceinline__ double pow2_neg(double d) { return (double)pow2_neg_f(d); }
-
 // part.y * 2^-(k_ch + mc) like chunk_contrib.  Partials that are zero, negative (never written) or carry an
 // infinite reference give exactly 0; a NaN sum stays NaN.
 __device__ __forceinline__ double scaled_contrib(float2 p, float c, double mc) {

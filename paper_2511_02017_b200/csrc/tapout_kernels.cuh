@@ -341,7 +341,8 @@ struct WalkShared {
     float2 gather[2][kMaxCluster][kWarps];   // per-warp (reference, sum) of every CTA of the cluster, by row parity
     double ctot[2][kMaxCluster];             // per-CTA totals of the final draw: [0] residual, [1] target row
     float2 wrec[kWarps];
-    double d0, d1;
+    double dm[2], dW[2];                     // the walk's row result (maximum, W) by row parity
+    int dec[2];                              // and its decision
     int i0, i1;
 };
 
@@ -365,8 +366,8 @@ __device__ __forceinline__ void gather_reduce(const WalkShared* sh, int par, int
     m = warp_max_f(fmaxf(r0.x, r1.x));
     const double mc = (double)m * (double)c;
     double w = 0.0;
-    if (r0.x != neg_inf() && r0.y > 0.f) w += (double)r0.y * exp2(-((double)__fmul_rn(-r0.x, c) + mc));
-    if (r1.x != neg_inf() && r1.y > 0.f) w += (double)r1.y * exp2(-((double)__fmul_rn(-r1.x, c) + mc));
+    if (r0.x != neg_inf() && r0.y > 0.f) w += (double)r0.y * pow2_neg((double)__fmul_rn(-r0.x, c) + mc);
+    if (r1.x != neg_inf() && r1.y > 0.f) w += (double)r1.y * pow2_neg((double)__fmul_rn(-r1.x, c) + mc);
     W = warp_sum_d(w);
     if (bad) W = (double)__int_as_float(0x7fc00000);
 }
@@ -455,13 +456,12 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
                     dec = (u24_to_double(w.x) < ratio) ? 1 : 0;
                 }
             }
-            if (lane == 0) { sh.i0 = dec; sh.d0 = (double)m; sh.d1 = W; }
+            if (lane == 0) { sh.dec[i & 1] = dec; sh.dm[i & 1] = (double)m; sh.dW[i & 1] = W; }
         }
-        __syncthreads();
-        const int dec = sh.i0;
-        m_p = (float)sh.d0;
-        W_p = sh.d1;
-        __syncthreads();
+        __syncthreads();                     // the slot of this parity is rewritten two rows on, behind a cluster barrier
+        const int dec = sh.dec[i & 1];
+        m_p = (float)sh.dm[i & 1];
+        W_p = sh.dW[i & 1];
         if (dec != 1) { acc_len = i; bad = dec < 0; break; }
     }
 
