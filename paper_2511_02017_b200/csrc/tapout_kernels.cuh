@@ -91,13 +91,14 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     const int pos = a.pos;
 
     // ---- first trip, everything at once: is the sequence drafting at this position, how many rows are
-    // (the split follows from it), all 64 segment-record slots (two per lane; those beyond the split are
+    // (the split follows from it), all segment-record slots (kMaxSeg / 32 per lane; those beyond the split are
     // stale and masked below), chunk partials, rule state.  Nothing here waits for anything else.
     const int np = FEATURES ? pos : __ldcg(sc.next_pos + s);
     const int n_rows = FEATURES ? a.n_fixed : __ldcg(sc.count + a.slot);
-    SegRec r[2];
+    constexpr int RPL = kMaxSeg / 32;        // segment records per lane
+    SegRec r[RPL];
 #pragma unroll
-    for (int j = 0; j < 2; ++j) r[j] = load_segrec(sc.seg + (size_t)s * kMaxSeg + lane + 32 * j);
+    for (int j = 0; j < RPL; ++j) r[j] = load_segrec(sc.seg + (size_t)s * kMaxSeg + lane + 32 * j);
     const bool in_regs = p.NC <= 32 * kRegPer;
     RegCdf cdf;
     if (in_regs) cdf.load(part, p.NC, lane);
@@ -118,12 +119,12 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     }
     const int nseg = segments_for(p, n_rows, n_warps_stream);
 #pragma unroll
-    for (int j = 0; j < 2; ++j)
+    for (int j = 0; j < RPL; ++j)
         if (lane + 32 * j >= nseg) { r[j].ref = neg_inf(); r[j].S = 0.f; r[j].T = 0.f; r[j].c2 = neg_inf(); r[j].best = -1; }
     bool has_nan = false;
     float m = neg_inf();
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
+    for (int j = 0; j < RPL; ++j) {
         has_nan = has_nan || (r[j].S != r[j].S) || (r[j].T != r[j].T) || (r[j].ref != r[j].ref);
         m = fmaxf(m, r[j].ref);
     }
@@ -132,7 +133,7 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     const double mc = (double)m * (double)c;
     double Tg = 0.0;
 #pragma unroll
-    for (int j = 0; j < 2; ++j)
+    for (int j = 0; j < RPL; ++j)
         if (r[j].ref > neg_inf() && r[j].ref < CUDART_INF_F) {
             const double d = (double)__fmul_rn(-r[j].ref, c) + mc;       // >= 0 up to rounding
             Tg += pow2_neg(d) * ((double)r[j].T - d * (double)r[j].S);
@@ -161,13 +162,22 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     }
 
     // ---- which chunk holds the maximum (the lowest such), which one the drawn token
-    const unsigned tie0 = __ballot_sync(0xffffffffu, r[0].best >= 0 && r[0].ref == m);
-    const unsigned tie1 = __ballot_sync(0xffffffffu, r[1].best >= 0 && r[1].ref == m);
-    const int win = tie0 ? __ffs(tie0) - 1 : 32 + __ffs(tie1) - 1;      // segments are in token order
-    const int best = max(__shfl_sync(0xffffffffu, win < 32 ? r[0].best : r[1].best, win & 31), 0);
-    const float other = warp_max_f(fmaxf(lane == win ? neg_inf() : r[0].ref, lane + 32 == win ? neg_inf() : r[1].ref));
-    const float c2all = warp_max_f(fmaxf(r[0].c2, r[1].c2));
-    const int n_tie = __popc(tie0) + __popc(tie1);
+    int win = -1, n_tie = 0, best = 0;                                   // segments are in token order
+    float other = neg_inf(), c2all = neg_inf();
+#pragma unroll
+    for (int j = 0; j < RPL; ++j) {
+        const unsigned tie = __ballot_sync(0xffffffffu, r[j].best >= 0 && r[j].ref == m);
+        n_tie += __popc(tie);
+        if (win < 0 && tie) {
+            win = 32 * j + __ffs(tie) - 1;
+            best = max(__shfl_sync(0xffffffffu, r[j].best, win & 31), 0);
+        }
+        c2all = fmaxf(c2all, r[j].c2);
+    }
+#pragma unroll
+    for (int j = 0; j < RPL; ++j) other = fmaxf(other, (lane + 32 * j == win) ? neg_inf() : r[j].ref);
+    other = warp_max_f(other);
+    c2all = warp_max_f(c2all);
     int chunk = 0;
     double rem = 0.0;
     float refc = 0.f;
