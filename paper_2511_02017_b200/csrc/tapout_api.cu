@@ -168,7 +168,7 @@ int setup_scratch(tapout* h) {
 // Chooses the arms of the coming round and sets up its lists; needed whenever no update ran since the
 // bandit statistics, the Philox inputs or the scratch memory last changed.
 int begin_round_now(tapout* h, int reset_adaedl) {
-    k_begin_round<<<(h->p.S + 3) / 4, 128, 0, h->stream>>>(h->p, h->st, h->sc, h->round, reset_adaedl);
+    k_begin_round<<<(unsigned)(((long long)h->p.S * h->p.P + 3) / 4), 128, 0, h->stream>>>(h->p, h->st, h->sc, h->round, reset_adaedl);
     TP_LAUNCHED(h);
     h->arms_ready = true;
     return TAPOUT_OK;
@@ -292,7 +292,7 @@ int update_impl(tapout* h) {
     if (!h) return TAPOUT_E_INVALID_ARG;
     if (!h->verified) return TAPOUT_E_BAD_STATE;
     { int rc = profile_mark(h, 2); if (rc) return rc; }
-    TP_CUDA(h, launch_chained(k_update, (unsigned)(h->p.S + 3) / 4, 128, 0, h->stream, 0, h->p, h->st, h->sc, h->round + 1));
+    TP_CUDA(h, launch_chained(k_update, (unsigned)(((long long)h->p.S * h->p.P + 3) / 4), 128, 0, h->stream, 0, h->p, h->st, h->sc, h->round + 1));
     TP_LAUNCHED(h);
     { int rc = profile_mark(h, 2); if (rc) return rc; }
     if (h->profile) h->prof_n[2] += 1;

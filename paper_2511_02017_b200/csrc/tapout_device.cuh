@@ -641,6 +641,20 @@ __device__ inline int ts_gauss_select(const Params& p, const uint32_t* N, const 
 __device__ inline uint32_t beta_order_stat_warp(const Params& p, uint32_t alpha, uint32_t beta, uint32_t seq,
                                                 uint32_t round, uint32_t pos, uint32_t arm, uint32_t* hist, int lane) {
     const uint32_t n = alpha + beta - 1;
+    if (n <= 32) {
+        // one uniform per lane; a lane's rank = uniforms below it, ties broken by lane, so ranks are distinct
+        const uint4 w = rng_words(p, seq, round, pos, RNG_BANDIT, arm, (uint32_t)lane >> 2);
+        const uint32_t sel = (uint32_t)lane & 3u;
+        const uint32_t mine = ((sel == 0) ? w.x : (sel == 1) ? w.y : (sel == 2) ? w.z : w.w) >> 8;
+        const bool have = (uint32_t)lane < n;
+        uint32_t rank = 0;
+        for (int l = 0; l < 32; ++l) {
+            const uint32_t other = __shfl_sync(0xffffffffu, mine, l);
+            rank += ((uint32_t)l < n) && (other < mine || (other == mine && l < lane));
+        }
+        const unsigned hit = __ballot_sync(0xffffffffu, have && rank == alpha - 1);
+        return __shfl_sync(0xffffffffu, mine, __ffs(hit) - 1);
+    }
     const uint32_t calls = (n + 3) / 4;
     uint32_t k = alpha - 1;                 // 0-based rank still to find among the candidates
     uint32_t prefix = 0;

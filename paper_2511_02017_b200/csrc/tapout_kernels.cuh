@@ -155,6 +155,7 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
             } else {
                 atomicOr(&sc.status[0], 1ull);
                 a.out_token[(size_t)s * a.tok_stride] = -1; a.out_continue[s] = 0; st.active[s] = 0;
+                if (pos == 0) st.n_drafted[s] = 0;       // nothing drafted this round (the update leaves the old length)
                 sc.stopped[atomicAdd(&sc.count[3], 1)] = s;
             }
         }
@@ -613,45 +614,36 @@ __device__ __forceinline__ int select_arm(const Params& p, const State& st, int 
     return __shfl_sync(0xffffffffu, arm, 0);
 }
 
-// Arms of round `round` for every sequence and slot, and the round's bookkeeping (one warp per sequence).
-__device__ __forceinline__ void begin_round(const Params& p, const State& st, const Scratch& sc, int s, uint32_t round,
-                                            uint32_t* hist, int lane) {
-    if (p.level == 0) {
-        const int arm = select_arm(p, st, s, 0, round, hist, lane);
-        for (int k = lane; k < p.K; k += 32) st.arm[(size_t)s * p.K + k] = arm;
-    } else if (p.policy == 1) {
-        for (int k = 0; k < p.K; ++k) {
-            const int arm = select_arm(p, st, s, k, round, hist, lane);
-            if (lane == 0) st.arm[(size_t)s * p.K + k] = arm;
-        }
-    } else {
-        // one lane per position; select_arm's scalar branch runs on lane 0 only, so call the scalar code directly
-        for (int k = lane; k < p.K; k += 32) {
-            const size_t o = ((size_t)s * p.P + k) * p.A;
-            st.arm[(size_t)s * p.K + k] = (p.policy == 0) ? ucb1_select(st.cnt + o, st.rsum + o, p.A, p.ucb_c2)
-                                                          : ucb_tuned_select(st.cnt + o, st.rsum + o, st.rsum2 + o, p.A);
-        }
-    }
-    if (lane == 0) {
-        st.active[s] = 1; st.n_drafted[s] = 0; st.sqrtH_prev[s] = 0.0;
-        sc.list[s] = s; sc.next_pos[s] = 0; sc.done[s] = 0;
+// Arm of round `round` for one bandit (sequence s, slot k; sequence level has the single slot 0, whose arm
+// serves every position), and, from the warp of slot 0, the round's bookkeeping.
+__device__ __forceinline__ void begin_round(const Params& p, const State& st, const Scratch& sc, int s, int k,
+                                            uint32_t round, uint32_t* hist, int lane, bool reset_counts) {
+    const int arm = select_arm(p, st, s, k, round, hist, lane);
+    if (p.level == 0) { for (int kk = lane; kk < p.K; kk += 32) st.arm[(size_t)s * p.K + kk] = arm; }
+    else if (lane == 0) st.arm[(size_t)s * p.K + k] = arm;
+    if (k == 0 && lane == 0) {
+        if (reset_counts) { st.active[s] = 1; st.n_drafted[s] = 0; st.sqrtH_prev[s] = 0.0; }
+        sc.list[s] = s; sc.next_pos[s] = 0;
         if (s == 0) { sc.count[0] = p.S; sc.count[1] = 0; sc.count[2] = 0; sc.count[3] = 0; }
     }
 }
 
-// update(pi, |Y|, |X|, gamma): rewards, arm statistics, AdaEDL; then the arms of the next round.
+// update(pi, |Y|, |X|, gamma): rewards, arm statistics, AdaEDL; then the arms of the next round.  One warp
+// per bandit (sequence, slot): the Beta draws of token-level Thompson Sampling cost O(plays) each, so the
+// slots of a sequence must not queue behind one another.  The drafted and accepted lengths are read by all
+// warps of a sequence and therefore left alone here: position 0 of the next round rewrites them.
 __global__ void __launch_bounds__(128)
 k_update(Params p, State st, Scratch sc, uint32_t next_round)
 {
     __shared__ uint32_t hist[4][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int s = blockIdx.x * 4 + warp;
+    const int gw = blockIdx.x * 4 + warp;
+    const int s = gw / p.P, k = gw - s * p.P;
     pdl_trigger();
     pdl_wait();
     if (s >= p.S) return;
     if (lane == 0) {
         const int n = st.n_drafted[s], a = st.accept_len[s];
-        double r_out = 0.0;
         if (n > 0) {
             if (p.level == 0) {
                 const double r = p.reward_kind ? ((double)a / (double)p.K)
@@ -659,27 +651,30 @@ k_update(Params p, State st, Scratch sc, uint32_t next_round)
                                                   (1.0 - p.reward_alpha) * ((double)a / (double)n));
                 const size_t o = (size_t)s * p.A + st.arm[(size_t)s * p.K];
                 st.cnt[o] += 1; st.rsum[o] += r; st.rsum2[o] += r * r;
-                r_out = r;
+                st.reward[s] = r;
             } else {
                 const int last = p.token_update_all ? n : min(a + 1, n);
-                for (int i = 0; i < last; ++i) {
-                    const double r = (i < a) ? 1.0 : 0.0;
-                    const size_t o = ((size_t)s * p.K + i) * p.A + st.arm[(size_t)s * p.K + i];
+                if (k < last) {
+                    const double r = (k < a) ? 1.0 : 0.0;
+                    const size_t o = ((size_t)s * p.K + k) * p.A + st.arm[(size_t)s * p.K + k];
                     st.cnt[o] += 1; st.rsum[o] += r; st.rsum2[o] += r * r;
                 }
-                r_out = (double)a;
+                if (k == 0) st.reward[s] = (double)a;
             }
-            // AdaEDL, as printed: lambda <- b2*lambda + (1-b2)*(lambda + eps*sign(alpha - r))
-            const double r = (double)a / (double)n;
-            const double d = p.ada_alpha - r;
-            const double sgn = (double)((d > 0.0) - (d < 0.0));
-            st.acc_rate[s] = p.ada_beta1 * st.acc_rate[s] + (1.0 - p.ada_beta1) * r;
-            st.lambda[s] = p.ada_beta2 * st.lambda[s] + (1.0 - p.ada_beta2) * (st.lambda[s] + p.ada_eps * sgn);
+            if (k == 0) {
+                // AdaEDL, as printed: lambda <- b2*lambda + (1-b2)*(lambda + eps*sign(alpha - r))
+                const double r = (double)a / (double)n;
+                const double d = p.ada_alpha - r;
+                const double sgn = (double)((d > 0.0) - (d < 0.0));
+                st.acc_rate[s] = p.ada_beta1 * st.acc_rate[s] + (1.0 - p.ada_beta1) * r;
+                st.lambda[s] = p.ada_beta2 * st.lambda[s] + (1.0 - p.ada_beta2) * (st.lambda[s] + p.ada_eps * sgn);
+            }
+        } else if (k == 0) {
+            st.reward[s] = 0.0;
         }
-        st.reward[s] = r_out;
     }
     __syncwarp();
-    begin_round(p, st, sc, s, next_round, hist[warp], lane);
+    begin_round(p, st, sc, s, k, next_round, hist[warp], lane, false);
 }
 
 // Start of a round without an update before it (a new handle, a changed parameter, restored state):
@@ -689,13 +684,14 @@ k_begin_round(Params p, State st, Scratch sc, uint32_t round, int reset_adaedl)
 {
     __shared__ uint32_t hist[4][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int s = blockIdx.x * 4 + warp;
+    const int gw = blockIdx.x * 4 + warp;
+    const int s = gw / p.P, k = gw - s * p.P;
     pdl_trigger();
     pdl_wait();
     if (s >= p.S) return;
-    if (reset_adaedl && lane == 0) { st.lambda[s] = p.ada_lambda0; st.acc_rate[s] = p.ada_acc0; }
+    if (reset_adaedl && k == 0 && lane == 0) { st.lambda[s] = p.ada_lambda0; st.acc_rate[s] = p.ada_acc0; }
     __syncwarp();
-    begin_round(p, st, sc, s, round, hist[warp], lane);
+    begin_round(p, st, sc, s, k, round, hist[warp], lane, true);
 }
 
 // After tapout_set_state in the middle of a round: the drafting list of position `pos` and the list of
