@@ -423,3 +423,35 @@ def test_round_call_matches_separate_calls():
     assert np.array_equal(a.get_state()["_blob"], b.get_state()["_blob"])
     a.destroy()
     b.destroy()
+
+
+def test_rounds_back_to_back_without_synchronising():
+    """Rounds enqueued with nothing between them (position 0 of a round then overlaps the previous round's
+    verification tail and update) give what the same rounds give with a synchronisation after every call."""
+    w = si.scaled(si.WORKLOADS["throughput"], n_seq=96, vocab=20008)
+    from tests.lockstep import make_device
+    a, b = make_device(w), make_device(w, token_out_stride=w.k_max)   # b's steps write column i of the token matrix
+    S, K, R = w.n_seq, w.k_max, 12
+    pool = [peaked_logits(w, r, DEV) for r in range(R)]
+    mk = lambda shape, dt: [torch.zeros(shape, dtype=dt, device=DEV) for _ in range(R)]
+    ta, ca, aa, na = mk((S, K), torch.int32), mk(S, torch.uint8), mk(S, torch.int32), mk(S, torch.int32)
+    tb, cb, ab, nb = mk((S, K), torch.int32), mk(S, torch.uint8), mk(S, torch.int32), mk(S, torch.int32)
+    torch.cuda.synchronize()
+    for r in range(R):                                   # nothing but launches
+        a.round(pool[r][0], pool[r][1], ta[r], ca[r], aa[r], na[r])
+    for r in range(R):
+        d, t = pool[r]
+        for i in range(K):
+            b.draft_step(d[:, i, :], tb[r][:, i], cb[r])
+            torch.cuda.synchronize()
+        b.verify(d, t, tb[r], ab[r], nb[r])
+        torch.cuda.synchronize()
+        b.update()
+        torch.cuda.synchronize()
+    torch.cuda.synchronize()
+    for r in range(R):
+        assert torch.equal(ta[r], tb[r]) and torch.equal(aa[r], ab[r]) and torch.equal(na[r], nb[r]), r
+    assert np.array_equal(a.get_state()["_blob"], b.get_state()["_blob"])
+    assert a.get_status() == b.get_status()
+    a.destroy()
+    b.destroy()
