@@ -147,7 +147,6 @@ int setup_scratch(tapout* h) {
     const size_t o_count = off;  off = align_up(off + sizeof(int32_t) * 8, 256);
     const size_t o_stop = off;   off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
     const size_t o_next = off;   off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
-    const size_t o_done = off;   off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
     const size_t o_status = off; off = align_up(off + sizeof(unsigned long long) * 4, 256);
     if (cudaMalloc(&h->d_scratch, off) != cudaSuccess) { cudaGetLastError(); return TAPOUT_E_ALLOC; }
     TP_CUDA(h, cudaMemsetAsync(h->d_scratch, 0, off, h->stream));
@@ -157,7 +156,6 @@ int setup_scratch(tapout* h) {
     h->sc.count = reinterpret_cast<int32_t*>(h->d_scratch + o_count);
     h->sc.stopped = reinterpret_cast<int32_t*>(h->d_scratch + o_stop);
     h->sc.next_pos = reinterpret_cast<int32_t*>(h->d_scratch + o_next);
-    h->sc.done = reinterpret_cast<int32_t*>(h->d_scratch + o_done);
     h->sc.status = reinterpret_cast<unsigned long long*>(h->d_scratch + o_status);
 
     h->grid_rows = h->n_sm * kResident;                       // persistent: every CTA resident
@@ -229,7 +227,7 @@ cudaError_t launch_chained(void (*kernel)(KArgs...), unsigned grid, unsigned blo
 StepArgs step_args(const tapout* h, const void* logits, int64_t stride, float c) {
     StepArgs a = {};
     a.logits = logits; a.row_stride = stride;
-    a.pos = h->pos; a.slot = h->pos % 3; a.n_fixed = -1; a.grid_ref = h->grid_rows;
+    a.pos = h->pos; a.slot = h->pos % 3; a.n_fixed = -1;
     a.round = h->round; a.c = c; a.inv_T = h->p.inv_Tq;
     a.tok_stride = 1;
     return a;
@@ -633,12 +631,12 @@ int tapout_row_stats(tapout_t* h, const void* logits, int n_rows, int64_t row_st
 
 // ---------------------------------------------------------------------------------------------
 // Allocation-free row statistics: the scratch of the feature pass in a fixed array of the library image.
-// Layout (bytes): segment records [rows][kMaxSeg], chunk partials [rows][chunks], per-row counters.
+// Layout (bytes): segment records [rows][kMaxSeg], chunk partials [rows][chunks], the work ticket.
 namespace {
 constexpr int kStaticMaxChunks = TAPOUT_STATIC_MAX_VOCAB / chunk_elems<DT_FP32>();     // fp32 chunks are the shorter ones
 constexpr size_t kStaticSegBytes = sizeof(SegRec) * TAPOUT_STATIC_MAX_ROWS * kMaxSeg;
 constexpr size_t kStaticCdfBytes = sizeof(float2) * (size_t)TAPOUT_STATIC_MAX_ROWS * kStaticMaxChunks;
-constexpr size_t kStaticDoneBytes = sizeof(int32_t) * (TAPOUT_STATIC_MAX_ROWS + 8);    // per-row counters, then `count`
+constexpr size_t kStaticDoneBytes = sizeof(int32_t) * 8;                               // the `count` words (work ticket)
 constexpr size_t kStaticBytes = kStaticSegBytes + kStaticCdfBytes + kStaticDoneBytes;
 }  // namespace
 
@@ -696,11 +694,10 @@ int tapout_row_stats_static(const void* logits, int n_rows, int vocab, int64_t r
     Scratch sc = {};
     sc.seg = reinterpret_cast<SegRec*>(d.base);
     sc.cdf = reinterpret_cast<float2*>(d.base + kStaticSegBytes);
-    sc.done = reinterpret_cast<int32_t*>(d.base + kStaticSegBytes + kStaticCdfBytes);
-    sc.count = sc.done + TAPOUT_STATIC_MAX_ROWS;
+    sc.count = reinterpret_cast<int32_t*>(d.base + kStaticSegBytes + kStaticCdfBytes);
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    // the per-row segment counters and the work ticket are the only part that has to start at zero
-    if (cudaMemsetAsync(sc.done, 0, kStaticDoneBytes, s) != cudaSuccess) { cudaGetLastError(); return TAPOUT_E_CUDA; }
+    // the work ticket is the only part that has to start at zero
+    if (cudaMemsetAsync(sc.count, 0, kStaticDoneBytes, s) != cudaSuccess) { cudaGetLastError(); return TAPOUT_E_CUDA; }
     StepArgs a = {};
     a.logits = logits; a.row_stride = row_stride; a.n_fixed = n_rows;
     a.c = c_of((float)inv_temp); a.inv_T = (float)inv_temp; a.tok_stride = 1; a.out_feat = out_features;

@@ -54,11 +54,10 @@ struct Scratch {
     SegRec* seg;                 // [S][kMaxSeg]
     float2* cdf;                 // [S][NC]: (reference logit, sum of 2^(z*c + k)) per chunk
     int32_t* list;               // [3][S] sequences drafting at position pos, in slot pos % 3
-    int32_t* count;              // [0..2] lengths of the three lists; [3] length of `stopped`; [4],[5] work tickets of
-                                 // the draft step by position parity; [6] work ticket of tapout_row_stats
+    int32_t* count;              // [0..2] lengths of the three lists; [3] length of `stopped`; [4] work ticket of the
+                                 // streaming kernel (zeroed by every finish kernel)
     int32_t* stopped;            // [S] sequences in the order in which they stopped drafting this round
     int32_t* next_pos;           // [S] position the sequence drafts at next (stays put once it has stopped)
-    int32_t* done;               // [S] segments of the sequence's current row already reduced
     unsigned long long* status;  // [0] sticky bits, [1] draft rows, [2] target rows, [3] residual rows
 };
 

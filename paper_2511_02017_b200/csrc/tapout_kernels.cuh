@@ -1,9 +1,11 @@
 // Kernels of libtapout (sm_100a).  The two streaming kernels read each needed logit row from HBM
 // exactly once with 128-bit coalesced loads; everything per-row that is scalar runs in double.
 //
-//   k_draft_step    one launch per draft position: a persistent grid strides over (row, segment)
-//                   items; the CTA that reduces the last segment of a row also finishes the row
-//                   (features, token draw, stop rule, bookkeeping), so no second launch is needed.
+//   k_draft_stream  first kernel of a draft position: a persistent grid of independent warps, each
+//                   reducing one segment of one drafted row (ticket-scheduled), leaving a segment
+//                   record and per-chunk partial sums.
+//   k_draft_finish  second kernel: one warp per sequence combines the segments of its row (features,
+//                   token draw, stop rule, bookkeeping, lists for the next position).
 //   k_verify_walk   one thread-block cluster per sequence: every CTA streams its slice of the target
 //                   row, the per-warp partial sums are exchanged through distributed shared memory,
 //                   and all CTAs take the same accept / reject decision before the next row.
@@ -55,7 +57,7 @@ __device__ __forceinline__ void stream_chunks(WarpAcc& acc, const void* row, int
 struct StepArgs {
     const void* logits;
     long long row_stride;
-    int pos, slot, n_fixed, grid_ref;
+    int pos, slot, n_fixed;
     uint32_t round;
     float c, inv_T;
     int32_t* out_token;
@@ -708,7 +710,6 @@ k_rebuild_lists(Params p, State st, Scratch sc, int pos)
     if (tid == 0) sh_n = 0;
     __syncthreads();
     for (int s = tid; s < p.S; s += blockDim.x) {
-        sc.done[s] = 0;
         if (st.active[s]) {
             sc.next_pos[s] = pos;
             sc.list[(size_t)slot * p.S + atomicAdd(&sh_n, 1)] = s;
