@@ -278,6 +278,7 @@ def bench_ours(args):
         dev.set_param("token_out_stride", 1)
         dev.round_host(hd, ht, o_tok, o_acc, o_nxt)                     # warm-up (allocates the staging buffers)
         se0 = dev.get_status()
+        ht0 = dev.get_host_traffic()
         if backend_ready:
             torch.distributed.barrier()
         torch.cuda.synchronize()
@@ -291,9 +292,10 @@ def bench_ours(args):
         rows_e_all, ms_e_all = aggregate(rows_e, dt * 1e3, world, backend_ready)
         e2e = {"value": rows_e_all / (ms_e_all * 1e-3), "unit": UNIT, "steps": e2e_steps,
                "ms_per_step": ms_e_all / e2e_steps,
-               "h2d_bytes_per_step": hd.numel() * hd.element_size() + ht.numel() * ht.element_size(),
-               "d2h_bytes_per_step": (o_tok.numel() + o_acc.numel() + o_nxt.numel()) * 4,
-               "api": "tapout_round_host (pinned host logits in, host tokens out)"}
+               "h2d_bytes_per_step": (dev.get_host_traffic()[0] - ht0[0]) / e2e_steps,
+               "d2h_bytes_per_step": (dev.get_host_traffic()[1] - ht0[1]) / e2e_steps,
+               "host_logits_bytes": hd.numel() * hd.element_size() + ht.numel() * ht.element_size(),
+               "api": "tapout_round_host (pinned host logits in, host tokens out; only the rows the method can need are copied)"}
 
     # ---- CPU oracle on a bounded sample of the same workload (rank 0, single-GPU runs only)
     cpu = None

@@ -210,15 +210,21 @@ int tapout_round(tapout_t* h, const void* draft_logits, const void* target_logit
                  uint8_t* out_continue, int32_t* out_accept_len, int32_t* out_next_token);
 
 /*
- * One whole round from HOST memory: copies the round's logits to the device,
- * runs k_max draft steps, verify and update, and copies the results back.
- * Blocks until done.  Host arrays: draft_logits [n_seq][k_max][vocab],
- * target_logits [n_seq][k_max+1][vocab] (contiguous), out_draft_tokens
- * int32 [n_seq][k_max] (-1 beyond the drafted length), out_accept_len and
- * out_next_token int32 [n_seq].  Device staging buffers are allocated on first use.
+ * One whole round from HOST memory: copies logits to the device, runs the draft steps, verify and
+ * update, and copies the results back.  Blocks until done.  Only rows the method can need are
+ * copied: per position the draft rows of the sequences still drafting (the continue flags are read
+ * back after every step, and the drafting ends when none is left), then target rows 0 .. n of
+ * every sequence (n = tokens it drafted).  Results and state are those of the separate calls.
+ * Host arrays (pinned memory makes the copies fast): draft_logits [n_seq][k_max][vocab],
+ * target_logits [n_seq][k_max+1][vocab] (contiguous), out_draft_tokens int32 [n_seq][k_max]
+ * (-1 beyond the drafted length), out_accept_len and out_next_token int32 [n_seq].  Device staging
+ * buffers are allocated on first use.
  */
 int tapout_round_host(tapout_t* h, const void* draft_logits, const void* target_logits,
                       int32_t* out_draft_tokens, int32_t* out_accept_len, int32_t* out_next_token);
+
+/* Bytes tapout_round_host has copied host-to-device and device-to-host so far (either pointer may be NULL). */
+int tapout_get_host_traffic(const tapout_t* h, uint64_t* h2d_bytes, uint64_t* d2h_bytes);
 
 /*
  * Table 1 features of arbitrary rows, outside any round (kernel-level checks and

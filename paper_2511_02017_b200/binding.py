@@ -36,7 +36,7 @@ _INT_PARAMS = {"seed", "dtype", "seq_offset", "step_row_stride", "q_seq_stride",
 EXPORTS = [
     "tapout_strerror", "tapout_last_cuda_error", "tapout_create", "tapout_destroy", "tapout_set_stream",
     "tapout_set_param_f64", "tapout_set_param_i64", "tapout_get_param_f64", "tapout_get_param_i64",
-    "tapout_set_arms", "tapout_draft_step", "tapout_verify", "tapout_update", "tapout_round", "tapout_round_host",
+    "tapout_set_arms", "tapout_draft_step", "tapout_verify", "tapout_update", "tapout_round", "tapout_round_host", "tapout_get_host_traffic",
     "tapout_row_stats", "tapout_row_stats_static", "tapout_state_bytes", "tapout_state_field", "tapout_get_state", "tapout_set_state",
     "tapout_get_round", "tapout_set_round", "tapout_get_status", "tapout_get_profile", "tapout_get_launch_count",
 ]
@@ -88,6 +88,7 @@ def load():
     L.tapout_update.argtypes = [vp]
     L.tapout_round.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     L.tapout_round_host.argtypes = [vp, vp, vp, vp, vp, vp]
+    L.tapout_get_host_traffic.argtypes = [vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     L.tapout_row_stats.argtypes = [vp, vp, i32, i64, dbl, vp]
     L.tapout_row_stats_static.argtypes = [vp, i32, i32, i64, i32, dbl, vp, vp]
     L.tapout_state_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
@@ -225,6 +226,11 @@ class Tapout:
                                              C.c_void_p(out_draft_tokens.data_ptr()),
                                              C.c_void_p(out_accept_len.data_ptr()),
                                              C.c_void_p(out_next_token.data_ptr())), "tapout_round_host")
+
+    def get_host_traffic(self):
+        a, b = C.c_uint64(), C.c_uint64()
+        self._check(self.L.tapout_get_host_traffic(self.h, C.byref(a), C.byref(b)), "tapout_get_host_traffic")
+        return a.value, b.value
 
     def row_stats(self, logits, n_rows, row_stride, inv_temp, out_features):
         self._check(self.L.tapout_row_stats(self.h, _dev_ptr(logits), n_rows, row_stride, float(inv_temp),

@@ -51,6 +51,8 @@ struct tapout {
     // host-round staging
     char* d_stage = nullptr;
     size_t stage_bytes = 0;
+    unsigned char* h_mask = nullptr;     // pinned: continue flags read back by tapout_round_host
+    uint64_t h2d_bytes = 0, d2h_bytes = 0;   // bytes tapout_round_host has moved
     uint64_t launches = 0;
     std::string cuda_err;
     int64_t tok_stride = 1;
@@ -382,6 +384,7 @@ int tapout_destroy(tapout_t* h) {
     if (h->d_state) cudaFree(h->d_state);
     if (h->d_scratch) cudaFree(h->d_scratch);
     if (h->d_stage) cudaFree(h->d_stage);
+    if (h->h_mask) cudaFreeHost(h->h_mask);
     delete h;
     return TAPOUT_OK;
 }
@@ -589,12 +592,50 @@ int tapout_round_host(tapout_t* h, const void* draft_logits, const void* target_
     uint8_t* d_cont = reinterpret_cast<uint8_t*>(d + o_cont);
     int32_t* d_acc = reinterpret_cast<int32_t*>(d + o_acc);
     int32_t* d_next = reinterpret_cast<int32_t*>(d + o_next);
+    if (!h->h_mask) {
+        if (cudaMallocHost(&h->h_mask, S) != cudaSuccess) { cudaGetLastError(); h->h_mask = nullptr; return TAPOUT_E_ALLOC; }
+    }
+    // Only the rows the method can need cross the bus: at each position the draft rows of the sequences
+    // still drafting (their continue flags come back after every step), then target rows 0 .. n of every
+    // sequence (n = tokens it drafted).  Rows go to their usual place in the staging tensors.
+    const char* hq = static_cast<const char*>(draft_logits);
+    const char* hp = static_cast<const char*>(target_logits);
+    const size_t rb = V * esz;                                            // bytes of one row
+    std::vector<int> active(S), n_drafted(S, 0);
+    for (size_t s2 = 0; s2 < S; ++s2) active[s2] = (int)s2;
     TP_CUDA(h, cudaMemsetAsync(d_tok, 0xff, 4 * S * K, h->stream));        // -1 beyond the drafted length
-    TP_CUDA(h, cudaMemcpyAsync(d + o_q, draft_logits, qb, cudaMemcpyHostToDevice, h->stream));
-    TP_CUDA(h, cudaMemcpyAsync(d + o_p, target_logits, pb, cudaMemcpyHostToDevice, h->stream));
-    for (int i = 0; i < p.K; ++i) {
-        int rc = draft_step_impl(h, d + o_q + (size_t)i * V * esz, (int64_t)(K * V), d_tok + i, (int64_t)K, d_cont);
+    for (int i = 0; i < p.K && !active.empty(); ++i) {
+        if (active.size() * 4 >= S) {                                     // most rows: one strided copy of the position
+            TP_CUDA(h, cudaMemcpy2DAsync(d + o_q + (size_t)i * rb, K * rb, hq + (size_t)i * rb, K * rb, rb, S,
+                                         cudaMemcpyHostToDevice, h->stream));
+            h->h2d_bytes += rb * S;
+        } else {
+            for (int s2 : active) {
+                const size_t o = ((size_t)s2 * K + i) * rb;
+                TP_CUDA(h, cudaMemcpyAsync(d + o_q + o, hq + o, rb, cudaMemcpyHostToDevice, h->stream));
+            }
+            h->h2d_bytes += rb * active.size();
+        }
+        int rc = draft_step_impl(h, d + o_q + (size_t)i * rb, (int64_t)(K * V), d_tok + i, (int64_t)K, d_cont);
         if (rc != TAPOUT_OK) return rc;
+        TP_CUDA(h, cudaMemcpyAsync(h->h_mask, d_cont, S, cudaMemcpyDeviceToHost, h->stream));
+        TP_CUDA(h, cudaStreamSynchronize(h->stream));
+        h->d2h_bytes += S;
+        std::vector<int> next;
+        for (int s2 : active) {
+            n_drafted[s2] = i + 1;
+            if (h->h_mask[s2]) next.push_back(s2);
+        }
+        active.swap(next);
+    }
+    // target rows 0 and 1 of every sequence in one strided copy, the further rows of longer drafts one by one
+    TP_CUDA(h, cudaMemcpy2DAsync(d + o_p, (K + 1) * rb, hp, (K + 1) * rb, 2 * rb, S, cudaMemcpyHostToDevice, h->stream));
+    h->h2d_bytes += 2 * rb * S;
+    for (size_t s2 = 0; s2 < S; ++s2) {
+        if (n_drafted[s2] < 2) continue;
+        const size_t o = (s2 * (K + 1) + 2) * rb, nb = (size_t)(n_drafted[s2] - 1) * rb;
+        TP_CUDA(h, cudaMemcpyAsync(d + o_p + o, hp + o, nb, cudaMemcpyHostToDevice, h->stream));
+        h->h2d_bytes += nb;
     }
     int rc = verify_impl(h, d + o_q, (int64_t)(K * V), (int64_t)V, d + o_p, (int64_t)((K + 1) * V), (int64_t)V, d_tok,
                          d_acc, d_next);
@@ -605,6 +646,14 @@ int tapout_round_host(tapout_t* h, const void* draft_logits, const void* target_
     TP_CUDA(h, cudaMemcpyAsync(out_accept_len, d_acc, 4 * S, cudaMemcpyDeviceToHost, h->stream));
     TP_CUDA(h, cudaMemcpyAsync(out_next_token, d_next, 4 * S, cudaMemcpyDeviceToHost, h->stream));
     TP_CUDA(h, cudaStreamSynchronize(h->stream));
+    h->d2h_bytes += 4 * S * K + 8 * S;
+    return TAPOUT_OK;
+}
+
+int tapout_get_host_traffic(const tapout_t* h, uint64_t* h2d_bytes, uint64_t* d2h_bytes) {
+    if (!h) return TAPOUT_E_INVALID_ARG;
+    if (h2d_bytes) *h2d_bytes = h->h2d_bytes;
+    if (d2h_bytes) *d2h_bytes = h->d2h_bytes;
     return TAPOUT_OK;
 }
 
