@@ -246,7 +246,7 @@ int draft_step_impl(tapout* h, const void* logits, int64_t stride, int32_t* out_
     // one event pair per round for all draft steps: opened here, closed when verify is called
     if (h->pos == 0) { int rc = profile_mark(h, 0); if (rc) return rc; }
     if (h->profile) h->prof_n[0] += 2;
-    const unsigned fin_grid = (unsigned)((h->p.S + 3) / 4);
+    const unsigned fin_grid = (unsigned)((2 * (long long)h->p.S + 3) / 4);    // two warps per sequence, four per CTA
     const int n_warps = h->grid_rows * kWarps;
     TP_CUDA(h, h->p.dtype == DT_BF16
                    ? launch_chained(k_draft_stream<DT_BF16, false>, h->grid_rows, kThreads, 0, h->stream, 0, h->p, h->sc, a)

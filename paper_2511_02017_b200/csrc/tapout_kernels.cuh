@@ -84,7 +84,10 @@ __device__ __forceinline__ void store_segrec(SegRec* g, const SegRec& r) {
 // the next position.  FEATURES (tapout_row_stats): the features only, nothing of the round's state is
 // touched.  Two dependent trips to memory: the segment records with the chunk partials (and the few
 // state words the rule needs), then the two 2 KB chunks that hold the row maximum and the drawn token.
-template <int DT, bool FEATURES>
+// ROLE: a draft row is finished by two warps that share nothing but their inputs: role 1 works out the
+// features, evaluates the stop rule and hands the sequence over, role 2 draws the token (both repeat the
+// cheap first part, the row total).  Role 0 does everything in one warp (FEATURES).
+template <int DT, bool FEATURES, int ROLE>
 __device__ __forceinline__ void finish_row(const Params& p, const State& st, const Scratch& sc, const StepArgs& a, int s,
                                            int n_warps_stream, int lane) {
     const char* row = reinterpret_cast<const char*>(a.logits) + (size_t)s * a.row_stride * Elem<DT>::BYTES;
@@ -106,17 +109,18 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     if (in_regs) cdf.load(part, p.NC, lane);
     int arm = 0;
     double sq_prev = 0.0, lambda = 0.0;
-    if (!FEATURES && lane == 0) {
+    if (!FEATURES && ROLE != 2 && lane == 0) {
         arm = st.arm[(size_t)s * p.K + pos];
         sq_prev = st.sqrtH_prev[s];
         lambda = st.lambda[s];
     }
     // the uniform of the token draw does not depend on anything loaded: worked out while the loads fly
     double u_draw = 0.0;
-    if (!FEATURES) u_draw = u24_to_double(rng_words(p, p.seq_offset + (uint32_t)s, a.round, (uint32_t)pos, RNG_DRAFT, 0, 0).x);
-    if (np != pos) {
+    if (!FEATURES && ROLE != 1) u_draw = u24_to_double(rng_words(p, p.seq_offset + (uint32_t)s, a.round, (uint32_t)pos, RNG_DRAFT, 0, 0).x);
+    // (role 1 may already have moved next_pos on to pos + 1 by the time role 2 looks)
+    if (ROLE == 2 ? np < pos : np != pos) {
         // stopped at an earlier position: drafts nothing
-        if (lane == 0 && np < pos) { a.out_token[(size_t)s * a.tok_stride] = -1; a.out_continue[s] = 0; }
+        if (ROLE != 2 && lane == 0 && np < pos) { a.out_token[(size_t)s * a.tok_stride] = -1; a.out_continue[s] = 0; }
         return;
     }
     const int nseg = segments_for(p, n_rows, n_warps_stream);
@@ -147,9 +151,9 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     else { tot = cdf_totals<true>(part, p.NC, c, mc, true, lane); W = tot.W; }
     const bool valid = !has_nan && (m > neg_inf()) && (m < CUDART_INF_F) && (W > 0.0) && (W < CUDART_INF);
 
-    if (!FEATURES && lane == 0) atomicAdd(&sc.status[1], 1ull);
+    if (!FEATURES && ROLE != 2 && lane == 0) atomicAdd(&sc.status[1], 1ull);
     if (!valid) {
-        if (lane == 0) {
+        if (ROLE != 2 && lane == 0) {
             if (FEATURES) {
                 float* fo = a.out_feat + (size_t)s * kFeat;
                 const float qn = __int_as_float(0x7fc00000);
@@ -168,7 +172,7 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     int win = -1, n_tie = 0, best = 0;                                   // segments are in token order
     float other = neg_inf(), c2all = neg_inf();
 #pragma unroll
-    for (int j = 0; j < RPL; ++j) {
+    for (int j = 0; j < (ROLE == 2 ? 0 : RPL); ++j) {
         const unsigned tie = __ballot_sync(0xffffffffu, r[j].best >= 0 && r[j].ref == m);
         n_tie += __popc(tie);
         if (win < 0 && tie) {
@@ -177,14 +181,16 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
         }
         c2all = fmaxf(c2all, r[j].c2);
     }
+    if (ROLE != 2) {
 #pragma unroll
-    for (int j = 0; j < RPL; ++j) other = fmaxf(other, (lane + 32 * j == win) ? neg_inf() : r[j].ref);
-    other = warp_max_f(other);
-    c2all = warp_max_f(c2all);
+        for (int j = 0; j < RPL; ++j) other = fmaxf(other, (lane + 32 * j == win) ? neg_inf() : r[j].ref);
+        other = warp_max_f(other);
+        c2all = warp_max_f(c2all);
+    }
     int chunk = 0;
     double rem = 0.0;
     float refc = 0.f;
-    if (!FEATURES) {
+    if (!FEATURES && ROLE != 1) {
         const double tgt = u_draw * W;
         if (in_regs) {
             chunk = cdf.locate(tgt, lane, c, mc, rem, refc);
@@ -195,8 +201,16 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     }
     // ---- second trip: both chunks on their way while the features are worked out
     uint4 vt[4], vx[4];
-    load_lane_block<DT>(row, p.V, best, lane, vt);
-    if (!FEATURES) load_lane_block<DT>(row, p.V, max(chunk, 0), lane, vx);
+    if (ROLE != 2) load_lane_block<DT>(row, p.V, best, lane, vt);
+    if (!FEATURES && ROLE != 1) load_lane_block<DT>(row, p.V, max(chunk, 0), lane, vx);
+    const float kch = __fmul_rn(-refc, c);
+    if (ROLE == 2) {
+        // x_i ~ softmax(row) inside the chunk, from the weights the streaming pass summed
+        int tok = -1;
+        if (chunk >= 0) tok = pick_softmax_block<DT>(vx, p.V, chunk, c, kch, rem * exp2((double)kch + mc), lane);
+        if (lane == 0) a.out_token[(size_t)s * a.tok_stride] = tok;
+        return;
+    }
 
     const float inv_T = FEATURES ? a.inv_T : p.inv_Tq;
     const double lw = log(W);
@@ -210,7 +224,6 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     scan_top_block<DT>(vt, p.V, best, m, lane, cnt, first, below);
     const float m2 = (n_tie >= 2 || cnt >= 2) ? m : fmaxf(fmaxf(other, c2all), below);
     // two exponentials from one call: lane 1 works out the scale of the token draw, the others p2
-    const float kch = __fmul_rn(-refc, c);
     const double ex = exp(lane == 1 ? kLn2 * ((double)kch + mc) : ((double)m2 - (double)m) * (double)inv_T);
     const double p2 = (m2 > neg_inf()) ? ex * p1 : 0.0;
     const double draw_scale = __shfl_sync(0xffffffffu, ex, 1);            // 2^(kch + mc)
@@ -247,10 +260,12 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
             sc.list[(size_t)nslot * p.S + atomicAdd(&sc.count[nslot], 1)] = s;
         }
     }
-    // x_i ~ softmax(row) inside the chunk, from the weights the streaming pass summed
-    int tok = -1;
-    if (chunk >= 0) tok = pick_softmax_block<DT>(vx, p.V, chunk, c, kch, rem * draw_scale, lane);
-    if (lane == 0) a.out_token[(size_t)s * a.tok_stride] = tok;
+    if (ROLE == 0) {
+        // x_i ~ softmax(row) inside the chunk, from the weights the streaming pass summed
+        int tok = -1;
+        if (chunk >= 0) tok = pick_softmax_block<DT>(vx, p.V, chunk, c, kch, rem * draw_scale, lane);
+        if (lane == 0) a.out_token[(size_t)s * a.tok_stride] = tok;
+    }
 }
 
 // ============================================================================================
@@ -315,7 +330,7 @@ k_draft_stream(Params p, Scratch sc, StepArgs a)
     if (first) pdl_wait();
 }
 
-// Second kernel of a draft position: one warp per sequence (finish_row; a sequence that is not drafting
+// Second kernel of a draft position: two warps per sequence (finish_row, roles 1 and 2; a sequence that is not drafting
 // at this position only gets its "nothing drafted" outputs), and the hand-over of the lists to the next
 // position.  n_warps_stream: warps of the k_draft_stream grid that cut the rows (the split is recomputed
 // alike).  FEATURES: rows 0 .. n_fixed-1.
@@ -332,8 +347,15 @@ k_draft_finish(Params p, State st, Scratch sc, StepArgs a, int n_warps_stream)
         sc.count[4] = 0;                                 // the work ticket of the next streaming kernel
         if (!FEATURES) sc.count[(a.slot + 2) % 3] = 0;   // the list two positions ahead is free again
     }
-    const int n = FEATURES ? a.n_fixed : p.S;
-    for (int s = gw; s < n; s += n_warps) finish_row<DT, FEATURES>(p, st, sc, a, s, n_warps_stream, lane);
+    if (FEATURES) {
+        for (int s = gw; s < a.n_fixed; s += n_warps) finish_row<DT, true, 0>(p, st, sc, a, s, n_warps_stream, lane);
+    } else {
+        // two warps per sequence: even warps the features and the rule, odd warps the token
+        for (int s = gw >> 1; s < p.S; s += n_warps >> 1) {
+            if (gw & 1) finish_row<DT, false, 2>(p, st, sc, a, s, n_warps_stream, lane);
+            else finish_row<DT, false, 1>(p, st, sc, a, s, n_warps_stream, lane);
+        }
+    }
 }
 
 // ============================================================================================
@@ -420,8 +442,11 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
     const int cid = blockIdx.x / CS;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    pdl_trigger();
+    // Wait first, then let the successors go: the streaming kernel of the next round's position 0 does not
+    // wait for its predecessors, so nothing after this kernel may start before the last finish kernel of
+    // this round (whose scratch position 0 overwrites) has completed.
     pdl_wait();
+    pdl_trigger();
     // longest drafts first: sequences still drafting, then the stopped ones, last stopped first
     const int n_act = sc.count[a.slot];
     const int s = (cid < n_act) ? sc.list[(size_t)a.slot * p.S + cid] : sc.stopped[p.S - 1 - cid];

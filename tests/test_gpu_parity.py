@@ -425,10 +425,11 @@ def test_round_call_matches_separate_calls():
     b.destroy()
 
 
-def test_rounds_back_to_back_without_synchronising():
+@pytest.mark.parametrize("n_seq,vocab", [(96, 20008), (7, 4104), (300, 2056)])
+def test_rounds_back_to_back_without_synchronising(n_seq, vocab):
     """Rounds enqueued with nothing between them (position 0 of a round then overlaps the previous round's
     verification tail and update) give what the same rounds give with a synchronisation after every call."""
-    w = si.scaled(si.WORKLOADS["throughput"], n_seq=96, vocab=20008)
+    w = si.scaled(si.WORKLOADS["throughput"], n_seq=n_seq, vocab=vocab)
     from tests.lockstep import make_device
     a, b = make_device(w), make_device(w, token_out_stride=w.k_max)   # b's steps write column i of the token matrix
     S, K, R = w.n_seq, w.k_max, 12
