@@ -147,7 +147,7 @@ int setup_scratch(tapout* h) {
     const size_t o_cdf = off;    off = align_up(off + sizeof(float2) * (size_t)p.S * p.NC, 256);
     const size_t o_list = off;   off = align_up(off + sizeof(int32_t) * 3 * (size_t)p.S, 256);
     const size_t o_count = off;  off = align_up(off + sizeof(int32_t) * 8, 256);
-    const size_t o_stop = off;   off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
+    const size_t o_stop = off;   off = align_up(off + sizeof(long long) * (size_t)p.S, 256);
     const size_t o_next = off;   off = align_up(off + sizeof(int32_t) * (size_t)p.S, 256);
     const size_t o_status = off; off = align_up(off + sizeof(unsigned long long) * 4, 256);
     if (cudaMalloc(&h->d_scratch, off) != cudaSuccess) { cudaGetLastError(); return TAPOUT_E_ALLOC; }
@@ -156,7 +156,7 @@ int setup_scratch(tapout* h) {
     h->sc.cdf = reinterpret_cast<float2*>(h->d_scratch + o_cdf);
     h->sc.list = reinterpret_cast<int32_t*>(h->d_scratch + o_list);
     h->sc.count = reinterpret_cast<int32_t*>(h->d_scratch + o_count);
-    h->sc.stopped = reinterpret_cast<int32_t*>(h->d_scratch + o_stop);
+    h->sc.stopped = reinterpret_cast<long long*>(h->d_scratch + o_stop);
     h->sc.next_pos = reinterpret_cast<int32_t*>(h->d_scratch + o_next);
     h->sc.status = reinterpret_cast<unsigned long long*>(h->d_scratch + o_status);
 
@@ -275,7 +275,7 @@ int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const vo
         return TAPOUT_E_ALIGNMENT;
     WalkArgs a = {};
     a.qlog = q; a.q_seq = q_seq; a.q_pos = q_pos; a.plog = pl; a.p_seq = p_seq; a.p_pos = p_pos;
-    a.toks = toks; a.slot = h->pos % 3; a.round = h->round;
+    a.toks = toks; a.slot = h->pos % 3; a.pos = h->pos; a.round = h->round;
     a.cq = c_of(h->p.inv_Tq); a.cp = c_of(h->p.inv_Tp);
     a.out_acc = out_acc; a.out_next = out_next;
     if (h->ev[0].size() % 2 == 1) { int rc = profile_mark(h, 0); if (rc) return rc; }

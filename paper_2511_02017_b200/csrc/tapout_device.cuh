@@ -56,7 +56,7 @@ struct Scratch {
     int32_t* list;               // [3][S] sequences drafting at position pos, in slot pos % 3
     int32_t* count;              // [0..2] lengths of the three lists; [3] length of `stopped`; [4] work ticket of the
                                  // streaming kernel (zeroed by every finish kernel)
-    int32_t* stopped;            // [S] sequences in the order in which they stopped drafting this round
+    long long* stopped;          // [S] (drafted length << 32 | sequence) in the order in which sequences stopped drafting
     int32_t* next_pos;           // [S] position the sequence drafts at next (stays put once it has stopped)
     unsigned long long* status;  // [0] sticky bits, [1] draft rows, [2] target rows, [3] residual rows
 };
@@ -136,6 +136,22 @@ template <> __device__ __forceinline__ float load_elem<DT_FP32>(const void* row,
 template <> __device__ __forceinline__ float load_elem<DT_BF16>(const void* row, int idx) {
     const uint32_t b = __ldg(reinterpret_cast<const unsigned short*>(row) + idx);
     return __uint_as_float(b << 16);
+}
+
+// Small asynchronous copies global -> shared (no register is held while they fly).
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// Element idx of a row, out of the aligned 32-bit word that holds it.
+template <int DT> __device__ __forceinline__ float word_elem(uint32_t w, int idx);
+template <> __device__ __forceinline__ float word_elem<DT_FP32>(uint32_t w, int) { return __uint_as_float(w); }
+template <> __device__ __forceinline__ float word_elem<DT_BF16>(uint32_t w, int idx) {
+    return __uint_as_float((idx & 1) ? (w & 0xffff0000u) : (w << 16));
 }
 
 // One warp chunk = 4 x 16 bytes per lane, lane-interleaved so every load instruction covers 512

@@ -54,6 +54,10 @@ __device__ __forceinline__ void stream_chunks(WarpAcc& acc, const void* row, int
 }
 
 // What the finishing warp needs besides Params / State / Scratch.
+// Entry of the list of stopped sequences: the sequence and the number of tokens it drafted, in one word, so
+// that the verification walk learns both from one load.
+__device__ __forceinline__ long long pack_stopped(int s, int n) { return ((long long)n << 32) | (unsigned)s; }
+
 struct StepArgs {
     const void* logits;
     long long row_stride;
@@ -162,7 +166,7 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
                 atomicOr(&sc.status[0], 1ull);
                 a.out_token[(size_t)s * a.tok_stride] = -1; a.out_continue[s] = 0; st.active[s] = 0;
                 if (pos == 0) st.n_drafted[s] = 0;       // nothing drafted this round (the update leaves the old length)
-                sc.stopped[atomicAdd(&sc.count[3], 1)] = s;
+                sc.stopped[atomicAdd(&sc.count[3], 1)] = pack_stopped(s, pos);       // drafted nothing here: length pos
             }
         }
         return;
@@ -253,7 +257,7 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
         st.active[s] = stop ? 0 : 1;
         a.out_continue[s] = stop ? 0 : 1;
         if (stop) {
-            sc.stopped[atomicAdd(&sc.count[3], 1)] = s;
+            sc.stopped[atomicAdd(&sc.count[3], 1)] = pack_stopped(s, pos + 1);
         } else {
             const int nslot = (a.slot + 1) % 3;
             sc.next_pos[s] = pos + 1;
@@ -367,16 +371,22 @@ struct WalkArgs {
     const void* plog; long long p_seq, p_pos;
     const int32_t* toks;
     int slot;                    // list of the sequences that were still drafting when verify was called
+    int pos;                     // draft steps taken this round = drafted length of those sequences
     uint32_t round;
     float cq, cp;
     int32_t* out_acc; int32_t* out_next;
 };
 
+constexpr int kWalkU = 32;
+
 struct WalkShared {
     float2 gather[2][kMaxCluster][kWarps];   // per-warp (reference, sum) of every CTA of the cluster, by row parity
     double ctot[2][kMaxCluster];             // per-CTA totals of the final draw: [0] residual, [1] target row
     float2 wrec[kWarps];
-    double dm[2], dW[2];                     // the walk's row result (maximum, W) by row parity
+    double dm[2], dW[2], dq[2];              // the walk's row result (maximum, W) and the draft row's lse, by row parity
+    double u[kWalkU];                        // uniforms of the accept tests of the first rows
+    uint32_t pw[2], qw[2];                   // the words holding z_p(x), z_q(x) of the row's draft token
+    int xs[2];                               // that token (-1: outside the vocabulary)
     int dec[2];                              // and its decision
     int i0, i1;
 };
@@ -449,8 +459,9 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
     pdl_trigger();
     // longest drafts first: sequences still drafting, then the stopped ones, last stopped first
     const int n_act = sc.count[a.slot];
-    const int s = (cid < n_act) ? sc.list[(size_t)a.slot * p.S + cid] : sc.stopped[p.S - 1 - cid];
-    const int n = st.n_drafted[s];
+    int s, n;
+    if (cid < n_act) { s = sc.list[(size_t)a.slot * p.S + cid]; n = a.pos; }
+    else { const long long e = sc.stopped[p.S - 1 - cid]; s = (int)(unsigned)e; n = (int)(e >> 32); }
     const uint32_t seq = p.seq_offset + (uint32_t)s;
     const char* pbase = reinterpret_cast<const char*>(a.plog) + (size_t)s * a.p_seq * ESZ;
     const char* qbase = reinterpret_cast<const char*>(a.qlog) + (size_t)s * a.q_seq * ESZ;
@@ -464,42 +475,62 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
     bool bad = false;
     float m_p = 0.f;
     double W_p = 0.0;
+    // What the accept test of a row needs besides the row's normaliser (the words holding z_p(x) and z_q(x),
+    // the draft row's lse) is copied to shared memory asynchronously while the row is streamed, by the last
+    // warp (the one with a chunk less when the slice does not divide evenly); it holds no registers.  The
+    // uniforms of the first rows are worked out up front by idle threads.
+    if (tid < n && tid < kWalkU) sh.u[tid] = u24_to_double(rng_words(p, seq, a.round, (uint32_t)tid, RNG_ACCEPT, 0, 0).x);
+    const bool helper = warp == kWarps - 1 && lane == 0;
+    int x_cur = -1;
+    if (helper && n > 0) x_cur = a.toks[(size_t)s * p.K];
+    double lse_q_rej = 0.0;
     for (int i = 0; i < n; ++i) {
         const char* prow = pbase + (size_t)i * a.p_pos * ESZ;
+        const int par = i & 1;
+        if (helper) {
+            const bool ok = x_cur >= 0 && x_cur < p.V;
+            sh.xs[par] = ok ? x_cur : -1;
+            if (ok) {
+                const size_t wo = ((size_t)x_cur * ESZ) & ~(size_t)3;         // the aligned word holding the element
+                cp_async4(&sh.pw[par], prow + wo);
+                cp_async4(&sh.qw[par], qbase + (size_t)i * a.q_pos * ESZ + wo);
+            }
+            cp_async8(&sh.dq[par], st.lse_q + (size_t)s * p.K + i);
+            if (i + 1 < n) x_cur = a.toks[(size_t)s * p.K + i + 1];
+        }
         WarpAcc acc;
         acc.init();
         stream_chunks<DT, false, false>(acc, prow, p.V, c0, c1, warp, lane, cp, [](int, float, float) {});
         const float Sw = warp_sum_f(acc.S);
-        gather_send(cl, &sh, i & 1, rank, CS, warp, lane, acc.ref, Sw);
+        gather_send(cl, &sh, par, rank, CS, warp, lane, acc.ref, Sw);
+        if (helper) cp_async_wait_all();
         cl.sync();
         if (warp == 0) {
             float m;
             double W;
-            gather_reduce(&sh, i & 1, CS, lane, cp, m, W);
+            gather_reduce(&sh, par, CS, lane, cp, m, W);
+            const int x = sh.xs[par];
             int dec;
             if (!(m > neg_inf()) || !(m < CUDART_INF_F) || !(W > 0.0) || !(W < CUDART_INF)) {
                 dec = -1;
+            } else if (x < 0) {
+                if (lane == 0 && rank == 0) atomicOr(&sc.status[0], 8ull);
+                dec = 0;
             } else {
-                const int x = a.toks[(size_t)s * p.K + i];
-                if (x < 0 || x >= p.V) {
-                    if (lane == 0 && rank == 0) atomicOr(&sc.status[0], 8ull);
-                    dec = 0;
-                } else {
-                    const char* qrow = qbase + (size_t)i * a.q_pos * ESZ;
-                    // p(x) / q(x) = exp((s_p(x) - m_p) - (s_q(x) - lse_q)) / W_p
-                    const double dp = ((double)load_elem<DT>(prow, x) - (double)m) * (double)p.inv_Tp;
-                    const double logq = (double)load_elem<DT>(qrow, x) * (double)p.inv_Tq - st.lse_q[(size_t)s * p.K + i];
-                    const double ratio = exp(dp - logq) / W;
-                    const uint4 w = rng_words(p, seq, a.round, (uint32_t)i, RNG_ACCEPT, 0, 0);
-                    dec = (u24_to_double(w.x) < ratio) ? 1 : 0;
-                }
+                const float zp = word_elem<DT>(sh.pw[par], x), zq = word_elem<DT>(sh.qw[par], x);
+                const double u = (i < kWalkU) ? sh.u[i] : u24_to_double(rng_words(p, seq, a.round, (uint32_t)i, RNG_ACCEPT, 0, 0).x);
+                // p(x) / q(x) = exp((s_p(x) - m_p) - (s_q(x) - lse_q)) / W_p
+                const double dp = ((double)zp - (double)m) * (double)p.inv_Tp;
+                const double logq = (double)zq * (double)p.inv_Tq - sh.dq[par];
+                dec = (u < exp(dp - logq) / W) ? 1 : 0;
             }
-            if (lane == 0) { sh.dec[i & 1] = dec; sh.dm[i & 1] = (double)m; sh.dW[i & 1] = W; }
+            if (lane == 0) { sh.dec[par] = dec; sh.dm[par] = (double)m; sh.dW[par] = W; }
         }
-        __syncthreads();                     // the slot of this parity is rewritten two rows on, behind a cluster barrier
-        const int dec = sh.dec[i & 1];
-        m_p = (float)sh.dm[i & 1];
-        W_p = sh.dW[i & 1];
+        __syncthreads();                     // the slots of this parity are rewritten two rows on, behind a cluster barrier
+        const int dec = sh.dec[par];
+        m_p = (float)sh.dm[par];
+        W_p = sh.dW[par];
+        lse_q_rej = sh.dq[par];
         if (dec != 1) { acc_len = i; bad = dec < 0; break; }
     }
 
@@ -514,7 +545,7 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
         // residual of the rejected slot: r = max(0, p - q), both rows in one pass (the target row is L2-hot)
         const char* qrow = qbase + (size_t)acc_len * a.q_pos * ESZ;
         const double lse_p = (double)m_p * (double)p.inv_Tp + log(W_p);
-        const double lse_q = st.lse_q[(size_t)s * p.K + acc_len];
+        const double lse_q = lse_q_rej;
         const float kp = (float)(-lse_p * kLog2e), kq = (float)(-lse_q * kLog2e);
         const double dp = (double)kp + lse_p * kLog2e, dq = (double)kq + lse_q * kLog2e;   // rounding left in kp, kq
         const float beta = (float)exp2(dq - dp);            // p = 2^(zc+kp) 2^-dp,  q = 2^(zc+kq) 2^-dq
@@ -754,7 +785,7 @@ k_rebuild_lists(Params p, State st, Scratch sc, int pos)
     }
     __syncthreads();
     for (int s = tid; s < p.S; s += blockDim.x)
-        if (!st.active[s]) sc.stopped[atomicAdd(&hist[min(max(st.n_drafted[s], 0), p.K)], 1)] = s;
+        if (!st.active[s]) sc.stopped[atomicAdd(&hist[min(max(st.n_drafted[s], 0), p.K)], 1)] = pack_stopped(s, st.n_drafted[s]);
 }
 
 }  // namespace tpo
