@@ -458,10 +458,10 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
     pdl_wait();
     pdl_trigger();
     // longest drafts first: sequences still drafting, then the stopped ones, last stopped first
+    const long long e = sc.stopped[p.S - 1 - cid];      // read alongside the count: almost always the one needed
     const int n_act = sc.count[a.slot];
-    int s, n;
+    int s = (int)(unsigned)e, n = (int)(e >> 32);
     if (cid < n_act) { s = sc.list[(size_t)a.slot * p.S + cid]; n = a.pos; }
-    else { const long long e = sc.stopped[p.S - 1 - cid]; s = (int)(unsigned)e; n = (int)(e >> 32); }
     const uint32_t seq = p.seq_offset + (uint32_t)s;
     const char* pbase = reinterpret_cast<const char*>(a.plog) + (size_t)s * a.p_seq * ESZ;
     const char* qbase = reinterpret_cast<const char*>(a.qlog) + (size_t)s * a.q_seq * ESZ;
