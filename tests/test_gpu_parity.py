@@ -218,6 +218,17 @@ def test_lockstep_full_size_sampled_sequences(name, rounds, n_sample):
     torch.cuda.empty_cache()
 
 
+def test_lockstep_full_size_many_rounds_sampled():
+    """The bench workload at full size over enough rounds for UCB1 to leave its exploration phase, with the
+    oracle following a handful of sequences."""
+    w = si.WORKLOADS["throughput"]
+    sample = sorted(np.random.default_rng(11).choice(w.n_seq, size=5, replace=False).tolist())
+    rep, dev, _ = run_lockstep(w, 30, sample=sample, device=DEV, check_state_every=5)
+    _assert_clean(rep, max_flip_rate=0.05)
+    dev.destroy()
+    torch.cuda.empty_cache()
+
+
 # ------------------------------------------------------------------ invalid rows, API misuse, state
 def test_unusable_rows_follow_the_oracle():
     S, V, K = 4, 2048, 4
