@@ -218,6 +218,16 @@ def test_lockstep_full_size_sampled_sequences(name, rounds, n_sample):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("dtype,vocab", [("bf16", 300008), ("fp32", 140004)])
+def test_vocabulary_beyond_the_register_resident_chunk_table(dtype, vocab):
+    """More than 256 chunks per row: the finish kernel searches the chunk partials in memory instead of registers."""
+    w = si.Workload("wide", 5, vocab, dtype, 3, 1, 5, "ucb1", "seq", seed=71)
+    rep, dev, _ = run_lockstep(w, 6, device=DEV, logits_fn=peaked_logits)
+    _assert_clean(rep)
+    dev.destroy()
+    torch.cuda.empty_cache()
+
+
 def test_lockstep_full_size_many_rounds_sampled():
     """The bench workload at full size over enough rounds for UCB1 to leave its exploration phase, with the
     oracle following a handful of sequences."""
