@@ -126,7 +126,7 @@ int setup_scratch(tapout* h) {
     if (p.nseg > p.NC) p.nseg = p.NC;
 
     // verify clusters: the requested size, reduced until the device can co-schedule such a cluster
-    int cs = h->cluster_user > 0 ? h->cluster_user : auto_cluster(p.NC, p.S, h->n_sm * kResident);
+    int cs = h->cluster_user > 0 ? h->cluster_user : auto_cluster(p.NC, p.S, h->n_sm * kWalkResident);
     if (cs > p.NC) cs = 1;
     for (;; cs >>= 1) {
         h->walk_smem = sizeof(float2) * (size_t)((p.NC + cs - 1) / cs + 1);

@@ -22,7 +22,8 @@ namespace cg = cooperative_groups;
 
 constexpr int kMaxCluster = 8;           // portable cluster size limit
 constexpr int kFinishThreads = 128;       // k_draft_finish: four rows per CTA, no register ceiling
-constexpr int kResident = 4;              // CTAs of a streaming kernel resident per SM (64 registers per thread)
+constexpr int kResident = 4;              // k_draft_stream CTAs resident per SM (64 registers per thread)
+constexpr int kWalkResident = 5;          // k_verify_walk CTAs resident per SM (48 registers: its fold keeps no entropy sums)
 
 // Into how many segments a draft row is cut, one warp per segment, decided on the device from the number
 // of rows actually drafted at this position (the host never learns it).  Many rows: about three items per
@@ -440,7 +441,7 @@ __device__ __forceinline__ int owner_locate(const WalkShared* sh, int which, int
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads, kResident)
+__global__ void __launch_bounds__(kThreads, kWalkResident)
 k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
 {
     constexpr int ESZ = Elem<DT>::BYTES;
