@@ -419,11 +419,13 @@ __device__ __forceinline__ void gather_reduce(const WalkShared* sh, int par, int
 }
 
 // Final draw, second half: the CTAs have exchanged their totals (ctot[which]); the CTA whose range holds
-// u * total locates the chunk among its own partials and returns it (others return -1).  Whole warp 0.
+// u * total locates the chunk among its own partials (t: their lane sums, kept from before the exchange)
+// and returns it (others return -1).  Whole warp 0.
 // total <= 0 gives chunk -2 on every CTA.
 template <bool SCALED>
 __device__ __forceinline__ int owner_locate(const WalkShared* sh, int which, int rank, int CS, const float2* sm_part,
-                                            int nloc, float c, double mc, double u, int lane, double& rem) {
+                                            int nloc, float c, double mc, double u, int lane, const CdfTotals& t,
+                                            double& rem) {
     double mine = 0.0;
     if (lane < CS) mine = sh->ctot[which][lane];
     const double incl = warp_incl_scan_d(mine, lane);
@@ -436,7 +438,6 @@ __device__ __forceinline__ int owner_locate(const WalkShared* sh, int which, int
     const int owner = over ? __ffs(over) - 1 : 31 - __clz(pos);
     const double before = __shfl_sync(0xffffffffu, incl - mine, owner);
     if (rank != owner) return -1;
-    const CdfTotals t = cdf_totals<false>(sm_part, nloc, c, mc, SCALED, lane);
     return cdf_locate<false>(sm_part, nloc, c, mc, SCALED, lane, t, tgt - before, rem);
 }
 
@@ -579,14 +580,15 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
             if (lane == 0) sm_part[ch - c0] = make_float2(0.f, tot);
         }
         __syncthreads();
+        CdfTotals t = {};
         if (warp == 0) {
-            const CdfTotals t = cdf_totals<false>(sm_part, nloc, 0.f, 0.0, false, lane);
+            t = cdf_totals<false>(sm_part, nloc, 0.f, 0.0, false, lane);
             if (lane < CS) cl.map_shared_rank(&sh, lane)->ctot[0][rank] = t.W;
         }
         cl.sync();
         if (warp == 0) {
             double rem;
-            const int lc = owner_locate<false>(&sh, 0, rank, CS, sm_part, nloc, 0.f, 0.0, u2, lane, rem);
+            const int lc = owner_locate<false>(&sh, 0, rank, CS, sm_part, nloc, 0.f, 0.0, u2, lane, t, rem);
             int tok = -1;
             if (lc >= 0) tok = pick_residual<DT>(prow, qrow, p.V, c0 + lc, cp, kp, cq, kq, beta, rem, lane);
             if (lane == 0) { sh.i0 = lc; sh.i1 = tok; }
@@ -614,22 +616,22 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
         cl.sync();                                           // also orders sm_part for warp 0
         bool ok = false;
         double mc = 0.0;
+        CdfTotals t = {};
         if (warp == 0) {
             float m;
             double W;
             gather_reduce(&sh, par, CS, lane, cp, m, W);
             ok = (m > neg_inf()) && (m < CUDART_INF_F) && (W > 0.0) && (W < CUDART_INF);
             mc = (double)m * (double)cp;
-            double Wc = 0.0;
-            if (ok) Wc = cdf_totals<false>(sm_part, nloc, cp, mc, true, lane).W;
-            if (lane < CS) cl.map_shared_rank(&sh, lane)->ctot[1][rank] = Wc;
+            if (ok) t = cdf_totals<false>(sm_part, nloc, cp, mc, true, lane);
+            if (lane < CS) cl.map_shared_rank(&sh, lane)->ctot[1][rank] = t.W;
         }
         cl.sync();
         if (warp == 0) {
             int lc = -2, tok = -1;
             if (ok) {
                 double rem;
-                lc = owner_locate<true>(&sh, 1, rank, CS, sm_part, nloc, cp, mc, u2, lane, rem);
+                lc = owner_locate<true>(&sh, 1, rank, CS, sm_part, nloc, cp, mc, u2, lane, t, rem);
                 if (lc >= 0) {
                     const float kch = __fmul_rn(-sm_part[lc].x, cp);
                     tok = pick_softmax<DT>(prow, p.V, c0 + lc, cp, kch, rem * exp2((double)kch + mc), lane);
