@@ -384,10 +384,11 @@ struct WalkShared {
     float2 gather[2][kMaxCluster][kWarps];   // per-warp (reference, sum) of every CTA of the cluster, by row parity
     double ctot[2][kMaxCluster];             // per-CTA totals of the final draw: [0] residual, [1] target row
     float2 wrec[kWarps];
-    double dm[2], dW[2], dq[2];              // the walk's row result (maximum, W) and the draft row's lse, by row parity
+    double dq[2];                            // the draft row's lse, by row parity
     double u[kWalkU];                        // uniforms of the accept tests of the first rows
     uint32_t pw[2], qw[2];                   // the words holding z_p(x), z_q(x) of the row's draft token
     int xs[2];                               // that token (-1: outside the vocabulary)
+    float kp, kq, beta;                      // constants of the residual pass after a rejection
     int dec[2];                              // and its decision
     int i0, i1;
 };
@@ -475,8 +476,6 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
     // ---- walk: accept x_i iff u_i < p_i(x_i) / q_i(x_i)
     int acc_len = n;
     bool bad = false;
-    float m_p = 0.f;
-    double W_p = 0.0;
     // What the accept test of a row needs besides the row's normaliser (the words holding z_p(x) and z_q(x),
     // the draft row's lse) is copied to shared memory asynchronously while the row is streamed, by the last
     // warp (the one with a chunk less when the slice does not divide evenly); it holds no registers.  The
@@ -485,7 +484,6 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
     const bool helper = warp == kWarps - 1 && lane == 0;
     int x_cur = -1;
     if (helper && n > 0) x_cur = a.toks[(size_t)s * p.K];
-    double lse_q_rej = 0.0;
     for (int i = 0; i < n; ++i) {
         const char* prow = pbase + (size_t)i * a.p_pos * ESZ;
         const int par = i & 1;
@@ -526,13 +524,18 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
                 const double logq = (double)zq * (double)p.inv_Tq - sh.dq[par];
                 dec = (u < exp(dp - logq) / W) ? 1 : 0;
             }
-            if (lane == 0) { sh.dec[par] = dec; sh.dm[par] = (double)m; sh.dW[par] = W; }
+            if (lane == 0) sh.dec[par] = dec;
+            if (dec == 0 && lane == 0) {
+                // rejected: the constants of the residual pass, once, for everybody
+                const double lse_p = (double)m * (double)p.inv_Tp + log(W), lse_q = sh.dq[par];
+                const float kp = (float)(-lse_p * kLog2e), kq = (float)(-lse_q * kLog2e);
+                const double dp = (double)kp + lse_p * kLog2e, dq = (double)kq + lse_q * kLog2e;   // rounding left in kp, kq
+                sh.kp = kp; sh.kq = kq;
+                sh.beta = (float)exp2(dq - dp);      // p = 2^(zc+kp) 2^-dp,  q = 2^(zc+kq) 2^-dq
+            }
         }
         __syncthreads();                     // the slots of this parity are rewritten two rows on, behind a cluster barrier
         const int dec = sh.dec[par];
-        m_p = (float)sh.dm[par];
-        W_p = sh.dW[par];
-        lse_q_rej = sh.dq[par];
         if (dec != 1) { acc_len = i; bad = dec < 0; break; }
     }
 
@@ -546,11 +549,7 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
     if (!bad && acc_len < n) {
         // residual of the rejected slot: r = max(0, p - q), both rows in one pass (the target row is L2-hot)
         const char* qrow = qbase + (size_t)acc_len * a.q_pos * ESZ;
-        const double lse_p = (double)m_p * (double)p.inv_Tp + log(W_p);
-        const double lse_q = lse_q_rej;
-        const float kp = (float)(-lse_p * kLog2e), kq = (float)(-lse_q * kLog2e);
-        const double dp = (double)kp + lse_p * kLog2e, dq = (double)kq + lse_q * kLog2e;   // rounding left in kp, kq
-        const float beta = (float)exp2(dq - dp);            // p = 2^(zc+kp) 2^-dp,  q = 2^(zc+kq) 2^-dq
+        const float kp = sh.kp, kq = sh.kq, beta = sh.beta;  // written with the rejecting decision
         for (int ch = c0 + warp; ch < c1; ch += kWarps) {
             uint4 vp[kVecPerLane], vq[kVecPerLane];
             load_chunk<DT>(prow, p.V, ch, lane, vp);
