@@ -68,6 +68,7 @@ def lib():
         L.orc_ts_beta_select.argtypes = [vp, vp, i32, u32, u32, u64, u32, u32, u32, vp]
         L.orc_verify_sequence.argtypes = [vp, C.c_long, vp, C.c_long, i32, i32, C.c_float, C.c_float,
                                           vp, i32, vp, u64, u32, u32, dbl, vp, C.POINTER(VerifyOut)]
+        L.orc_verify_sequence_greedy.argtypes = [vp, C.c_long, i32, i32, C.c_float, vp, i32, C.POINTER(VerifyOut)]
         L.orc_create.restype = vp
         L.orc_create.argtypes = [i32] * 6
         L.orc_destroy.argtypes = [vp]
@@ -212,6 +213,17 @@ def verify_sequence(q_rows, p_rows, x, lse_q, seed, seq, rnd, inv_Tq=1.0, inv_Tp
     lib().orc_verify_sequence(_ptr(q_rows), V, _ptr(p_rows), V, _dtype_code(p_rows), V,
                               np.float32(inv_Tq), np.float32(inv_Tp), _ptr(x), x.shape[0], _ptr(lse_q),
                               seed, seq, rnd, tol, _ptr(scratch), C.byref(out))
+    return out
+
+
+def verify_sequence_greedy(p_rows, x, inv_Tp=1.0):
+    """Verification by matching the target's top-ranked token.  p_rows [>= n+1][V], x [n] tokens."""
+    p_rows = np.ascontiguousarray(p_rows)
+    x = np.ascontiguousarray(x, dtype=np.int32)
+    V = p_rows.shape[1]
+    out = VerifyOut()
+    lib().orc_verify_sequence_greedy(_ptr(p_rows), V, _dtype_code(p_rows), V, np.float32(inv_Tp), _ptr(x), x.shape[0],
+                                     C.byref(out))
     return out
 
 

@@ -454,6 +454,34 @@ void orc_verify_sequence(const void* q_rows, long q_pos_stride, const void* p_ro
 }
 
 /* ------------------------------------------------------------------------- */
+/* Verification read literally (Algorithm 1: "accept maximal matching prefix"; */
+/* Section 2: the target accepts the drafted tokens "that match its           */
+/* predictions"): the target's prediction at slot i is the token it ranks     */
+/* first, argmax_v p_i(v) (lowest index among equal maxima); x_i is accepted   */
+/* iff it is that token.  The final token is the target's own prediction at    */
+/* the first mismatching slot, or at slot n when everything matched.  No       */
+/* random numbers; rows after the first mismatch are not read.                 */
+/* ------------------------------------------------------------------------- */
+void orc_verify_sequence_greedy(const void* p_rows, long p_pos_stride, int dtype, int V, float inv_Tp,
+                                const int32_t* x, int n, orc_verify_out* out)
+{
+    size_t esz = (dtype == ORC_FP32) ? 4 : 2;
+    memset(out, 0, sizeof *out);
+    out->next_token = -1; out->next_lo = -1; out->next_hi = -1;
+    out->accept_len = n;
+    for (int i = 0; i <= n; ++i) {
+        const void* prow = (const char*)p_rows + (size_t)i * p_pos_stride * esz;
+        orc_rowstats sp;
+        if (!orc_row_stats(prow, dtype, V, inv_Tp, NULL, &sp)) { out->bad_target = 1; out->accept_len = i; return; }
+        if (i == n || x[i] != sp.argmax) {              /* first mismatch, or the slot after a full match */
+            out->accept_len = i;
+            out->next_token = out->next_lo = out->next_hi = sp.argmax;
+            return;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------- */
 /* The round engine: Algorithm 1 over a batch of independent sequences.      */
 /* ------------------------------------------------------------------------- */
 typedef struct {
@@ -472,6 +500,8 @@ typedef struct {
     uint32_t ts_beta_a0, ts_beta_b0;
     double ada_lambda0, ada_acc0;
     int token_update_all;        /* 1: every drafted position gets r_i = [i <= a]; 0: only i <= a+1 */
+    int draft_greedy;            /* 1: x_i = argmax q_i instead of a draw                        */
+    int verify_greedy;           /* 1: verification by matching the target's argmax (see above)  */
     double tol;                  /* near-threshold band, 1e-6 */
     /* per-sequence global ids (RNG stream of local sequence s is seq_id[s]) */
     uint32_t* seq_id;
@@ -622,10 +652,11 @@ int orc_draft_step(orc_t* h, const void* logits, long row_stride,
         f[0] = st.m; f[1] = st.lse; f[2] = st.p1; f[3] = st.p2; f[4] = st.H; f[5] = (double)st.argmax;
         h->lse_q[(size_t)s * h->K + i] = st.lse;
 
-        /* x_i ~ M_q */
+        /* x_i ~ M_q (greedy decoding of the draft: its most probable token) */
         double u = orc_rng_uniform(h->seed, h->seq_id[s], h->round, (uint32_t)i, ORC_RNG_DRAFT, 0, 0, 0);
         int lo, hi;
-        out_token[s] = orc_sample_cdf(w, h->V, st.W, u, h->tol, &lo, &hi);
+        if (h->draft_greedy) out_token[s] = lo = hi = st.argmax;
+        else out_token[s] = orc_sample_cdf(w, h->V, st.W, u, h->tol, &lo, &hi);
         if (tok_lo) tok_lo[s] = lo;
         if (tok_hi) tok_hi[s] = hi;
         free(w);
@@ -663,15 +694,19 @@ int orc_verify(orc_t* h, const void* draft_logits, long q_seq_stride, long q_pos
         double* scratch = (double*)malloc(sizeof(double) * 3 * (size_t)h->V);
         orc_verify_out vo;
         int n = h->n_drafted[s];
-        orc_verify_sequence((const char*)draft_logits + (size_t)s * q_seq_stride * esz, q_pos_stride,
-                            (const char*)target_logits + (size_t)s * p_seq_stride * esz, p_pos_stride,
-                            h->dtype, h->V, h->inv_Tq, h->inv_Tp,
-                            draft_tokens + (size_t)s * h->K, n, h->lse_q + (size_t)s * h->K,
-                            h->seed, h->seq_id[s], h->round, h->tol, scratch, &vo);
+        if (h->verify_greedy)
+            orc_verify_sequence_greedy((const char*)target_logits + (size_t)s * p_seq_stride * esz, p_pos_stride,
+                                       h->dtype, h->V, h->inv_Tp, draft_tokens + (size_t)s * h->K, n, &vo);
+        else
+            orc_verify_sequence((const char*)draft_logits + (size_t)s * q_seq_stride * esz, q_pos_stride,
+                                (const char*)target_logits + (size_t)s * p_seq_stride * esz, p_pos_stride,
+                                h->dtype, h->V, h->inv_Tq, h->inv_Tp,
+                                draft_tokens + (size_t)s * h->K, n, h->lse_q + (size_t)s * h->K,
+                                h->seed, h->seq_id[s], h->round, h->tol, scratch, &vo);
         free(scratch);
         if (vo.bad_target) status |= ORC_ST_BAD_TARGET_ROW;
         if (vo.zero_residual) status |= ORC_ST_ZERO_RESIDUAL;
-        rows += (uint64_t)vo.accept_len + 1 + (vo.accept_len < n ? 1 : 0);
+        rows += (uint64_t)vo.accept_len + 1 + ((vo.accept_len < n && !h->verify_greedy) ? 1 : 0);
         h->accept_len[s] = vo.accept_len;
         out_accept_len[s] = vo.accept_len;
         out_next_token[s] = vo.next_token;
@@ -755,6 +790,8 @@ int orc_set_param(orc_t* h, const char* key, double v)
     else if (K_("ts_beta_a0")) h->ts_beta_a0 = (uint32_t)v;
     else if (K_("ts_beta_b0")) h->ts_beta_b0 = (uint32_t)v;
     else if (K_("token_update_all")) h->token_update_all = (int)v;
+    else if (K_("draft_greedy")) h->draft_greedy = (int)v;
+    else if (K_("verify_greedy")) h->verify_greedy = (int)v;
     else if (K_("tol")) h->tol = v;
     else return -1;
 #undef K_

@@ -1,0 +1,153 @@
+"""Pins for the oracle's greedy variant: verification read literally as "accept the maximal matching
+prefix" (Algorithm 1; Section 2: tokens "that match its predictions"), and the draft's greedy decoding.
+
+The target's prediction at a slot is the token it ranks first.  Pinned by: numpy's argmax (first
+occurrence) on random rows with a planted mismatch; tie and early-exit cases built by hand; and the limit
+in which speculative sampling itself turns into prefix matching (a target distribution that puts all its
+mass on one token accepts exactly that token and resamples exactly that token)."""
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_2511_02017_b200.synth_inputs import bf16_bits_from_float
+
+
+def _rows(rng, n_rows, V, dtype):
+    z = (rng.normal(size=(n_rows, V)) * 3).astype(np.float32)
+    if dtype == "bf16":
+        bits = bf16_bits_from_float(z)
+        return bits, (bits.astype(np.uint32) << 16).view(np.float32)
+    return z, z
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("V", [5, 37, 1030])
+def test_matching_prefix_against_numpy_argmax(dtype, V):
+    rng = np.random.default_rng(V)
+    for trial in range(60):
+        n = int(rng.integers(1, 9))
+        rows, vals = _rows(rng, n + 1, V, dtype)
+        top = vals.argmax(axis=1)                       # first occurrence of the maximum
+        j = int(rng.integers(0, n + 1))                 # first mismatching slot; n = none
+        x = top[:n].copy()
+        if j < n:
+            x[j] = (top[j] + 1 + rng.integers(0, V - 1)) % V
+            x[j + 1:] = rng.integers(0, V, n - j - 1)   # whatever follows is never looked at
+        out = orc.verify_sequence_greedy(rows, x, inv_Tp=1.0 if trial % 2 else 1 / 0.7)
+        assert out.accept_len == j
+        assert out.next_token == top[j]                 # the target's own token at the first mismatch / the extra slot
+        assert not out.bad_target and not out.zero_residual and not out.near_accept
+
+
+def test_equal_maxima_predict_the_lowest_index():
+    row = np.zeros(12, np.float32)
+    row[[3, 7]] = 5.0
+    P = np.stack([row, row, row])
+    assert orc.verify_sequence_greedy(P, [7, 3]).accept_len == 0          # 7 is not the prediction
+    out = orc.verify_sequence_greedy(P, [3, 3])
+    assert (out.accept_len, out.next_token) == (2, 3)
+    # bf16 rounding makes ties common: 1.0 and 1.001 are the same bf16 number
+    bits = bf16_bits_from_float(np.array([[0.5, 1.001, 1.0, 0.2]], np.float32))
+    assert orc.verify_sequence_greedy(bits, []).next_token == 1
+
+
+def test_rows_behind_the_first_mismatch_are_not_read_and_bad_rows_end_the_walk():
+    rng = np.random.default_rng(3)
+    V, n = 40, 5
+    rows, vals = _rows(rng, n + 1, V, "fp32")
+    top = vals.argmax(axis=1)
+    x = top[:n].copy()
+    x[2] = (top[2] + 1) % V
+    poisoned = rows.copy()
+    poisoned[3:] = np.nan
+    out = orc.verify_sequence_greedy(poisoned, x)
+    assert (out.accept_len, out.next_token, out.bad_target) == (2, top[2], 0)
+    poisoned = rows.copy()
+    poisoned[1, 9] = np.nan                              # a needed row with a NaN
+    out = orc.verify_sequence_greedy(poisoned, x)
+    assert (out.accept_len, out.next_token, out.bad_target) == (1, -1, 1)
+    masked = rows.copy()
+    masked[0] = -np.inf                                  # no finite maximum
+    assert orc.verify_sequence_greedy(masked, x).bad_target == 1
+    masked = rows.copy()
+    masked[0, top[0]] = -np.inf                          # a masked token is never the prediction
+    out = orc.verify_sequence_greedy(masked, x)
+    assert out.accept_len == 0 and out.next_token == np.argmax(masked[0])
+
+
+def test_speculative_sampling_with_a_one_token_target_is_prefix_matching():
+    """p_i = delta(t_i): min(1, p/q) accepts x_i = t_i with certainty and rejects anything else with
+    certainty; the residual max(0, p - q) and the extra row's distribution both sit on t alone."""
+    rng = np.random.default_rng(4)
+    V, n = 30, 6
+    for seq in range(150):
+        zq = (rng.normal(size=(n, V)) * 2).astype(np.float32)
+        t = rng.integers(0, V, n + 1)
+        zp = np.full((n + 1, V), -np.inf, np.float32)
+        zp[np.arange(n + 1), t] = 0.0
+        x = t[:n].copy()
+        j = int(rng.integers(0, n + 1))
+        if j < n:
+            x[j] = (t[j] + 1 + rng.integers(0, V - 1)) % V
+        lse = [orc.row_stats(zq[i]).lse for i in range(n)]
+        a = orc.verify_sequence(zq, zp, x, lse, seed=9, seq=seq, rnd=1)
+        g = orc.verify_sequence_greedy(zp, x)
+        assert (a.accept_len, a.next_token) == (g.accept_len, g.next_token) == (j, t[j])
+
+
+def _engine(V, K, S, **params):
+    return orc.Oracle(S, V, K, 5, orc.UCB1, orc.SEQ, dtype=orc.FP32, seed=5, **params)
+
+
+def test_greedy_draft_token_is_the_argmax_and_leaves_the_features_alone():
+    rng = np.random.default_rng(6)
+    S, V, K = 9, 300, 4
+    z = (rng.normal(size=(S, V)) * 3).astype(np.float32)
+    z[2, [10, 200]] = 12.0                               # duplicated maximum
+    a, b = _engine(V, K, S), _engine(V, K, S, draft_greedy=1)
+    ra, rb = a.draft_step(z), b.draft_step(z)
+    assert np.array_equal(rb["token"], z.argmax(axis=1))
+    assert rb["token"][2] == 10
+    assert np.array_equal(ra["cont"], rb["cont"])                 # the stop rule sees the same features
+    assert np.array_equal(a.view("feat")[:, 0], b.view("feat")[:, 0])
+    assert not np.array_equal(ra["token"], rb["token"])                   # the draw does not always hit the mode
+
+
+def test_greedy_round_with_identical_models_accepts_everything():
+    rng = np.random.default_rng(7)
+    S, V, K = 6, 120, 5
+    o = _engine(V, K, S, draft_greedy=1, verify_greedy=1)
+    for rnd in range(4):
+        T = (rng.normal(size=(S, K + 1, V)) * 3).astype(np.float32)
+        D = T[:, :K].copy()
+        toks = np.full((S, K), -1, np.int32)
+        for i in range(K):
+            toks[:, i] = o.draft_step(D[:, i])["token"]
+        n = o.view("n_drafted").copy()
+        rows0 = o.rows_read
+        v = o.verify(D, T, toks)
+        assert np.array_equal(v["accept_len"], n)
+        assert np.array_equal(v["next_token"], T[np.arange(S), n].argmax(axis=1))
+        assert o.rows_read - rows0 == int((n + 1).sum())                   # a + 1 target rows, no residual row
+        o.update()
+        assert np.allclose(o.view("reward"), 0.5 * n / K + 0.5)           # r_blend with a = n
+    assert o.status == 0
+
+
+def test_greedy_round_counts_rows_and_rewards_on_a_mismatch():
+    S, V, K = 1, 50, 4
+    o = orc.Oracle(S, V, K, 1, orc.UCB1, orc.SEQ, dtype=orc.FP32, seed=1, arms=[orc.RULE_STATIC], draft_greedy=1,
+                   verify_greedy=1)
+    rng = np.random.default_rng(8)
+    T = (rng.normal(size=(S, K + 1, V)) * 3).astype(np.float32)
+    D = T[:, :K].copy()
+    D[0, 2, T[0, 2].argmax()] = -50.0                    # the draft disagrees at slot 2
+    toks = np.full((S, K), -1, np.int32)
+    for i in range(K):
+        toks[:, i] = o.draft_step(D[:, i])["token"]
+    rows0 = o.rows_read
+    v = o.verify(D, T, toks)
+    assert v["accept_len"][0] == 2 and v["next_token"][0] == T[0, 2].argmax()
+    assert o.rows_read - rows0 == 3
+    o.update()
+    assert o.view("reward")[0] == 0.5 * 2 / 4 + 0.5 * 2 / 4
