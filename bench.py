@@ -152,12 +152,21 @@ def run_round(dev, w, draft, target, toks, cont, acc, nxt):
     dev.round(draft, target, toks, cont, acc, nxt)
 
 
-def oracle_sample(w, draft, target, n_seq_sample, rounds, seq_offset=0):
+VARIANT_NOTE = "; greedy variant (draft argmax, verification by matching the target's top token)"
+
+
+def variant_params(args):
+    """--greedy: the literal reading of the verification step (match the target's top token) with a greedily
+    decoding draft, on both arms."""
+    return dict(draft_greedy=1, verify_greedy=1) if args.greedy else {}
+
+
+def oracle_sample(w, draft, target, n_seq_sample, rounds, seq_offset=0, params=None):
     """Times the oracle, as it stands, on `n_seq_sample` sequences of the given rounds' logits."""
     from oracle import oracle as orc
     from tests.lockstep import make_oracle
     ids = np.arange(n_seq_sample)
-    ora = make_oracle(w, ids + seq_offset)
+    ora = make_oracle(w, ids + seq_offset, **(params or {}))
     K = w.k_max
     hosts = [(si.to_numpy_bits(d[:n_seq_sample]), si.to_numpy_bits(t[:n_seq_sample])) for d, t in zip(draft, target)]
     t0 = time.perf_counter()
@@ -190,7 +199,7 @@ def bench_ours(args):
     POOL_ROUNDS = args.pool_rounds
     S, K, V = w.n_seq, w.k_max, w.vocab
     # weak scaling: every rank owns a full-size shard of independent sequences, ids offset by rank
-    dev = tp.Tapout.from_workload(w, seq_offset=rank * S, token_out_stride=K)
+    dev = tp.Tapout.from_workload(w, seq_offset=rank * S, token_out_stride=K, **variant_params(args))
     if args.row_segments:
         dev.set_param("row_segments", args.row_segments)
     if args.verify_cluster:
@@ -255,7 +264,7 @@ def bench_ours(args):
         ms_k, n_k = prof[k]
         return {"launches": n_k, "ms_total": ms_k, "alg_bytes": rows_k * row_bytes,
                 "gbs": rows_k * row_bytes / (ms_k * 1e-3) / 1e9 if ms_k > 0 else None}
-    kernels = {"k_draft_stream+k_draft_finish": kinfo(0, d_rows), "k_verify_walk": kinfo(1, v_rows),
+    kernels = {"k_draft_stream+k_draft_finish": kinfo(0, d_rows), ("k_verify_greedy" if args.greedy else "k_verify_walk"): kinfo(1, v_rows),
                "k_update": kinfo(2, 0)}
     dom = max(kernels, key=lambda k: kernels[k]["ms_total"])
     achieved = kernels[dom]["gbs"] or 0.0
@@ -301,7 +310,7 @@ def bench_ours(args):
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         n_s = min(S, args.cpu_sample_seqs)
-        rows_o, dt_o, cores = oracle_sample(w, [pool[0][0]], [pool[0][1]], n_s, args.cpu_sample_rounds)
+        rows_o, dt_o, cores = oracle_sample(w, [pool[0][0]], [pool[0][1]], n_s, args.cpu_sample_rounds, params=variant_params(args))
         cpu = {"value": rows_o / dt_o, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": "%d of %d sequences, %d round(s) of this workload's logits, %d rows in %.1f s" %
                          (n_s, S, args.cpu_sample_rounds, rows_o, dt_o)}
@@ -312,8 +321,8 @@ def bench_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_all / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": "%s: batch %d, vocab %d, %s logits, k_max %d, %s-level %s, %d arms" %
-                                   (w.name, S, V, w.dtype, K, w.level, w.policy, w.n_arms),
+            "config": {"workload": "%s: batch %d, vocab %d, %s logits, k_max %d, %s-level %s, %d arms%s" %
+                                   (w.name, S, V, w.dtype, K, w.level, w.policy, w.n_arms, VARIANT_NOTE if args.greedy else ""),
                        "rows_per_step": rows / args.steps, "row_bytes": row_bytes,
                        "l2_policy": "inputs larger than L2: %d rounds of %.2f GB cycled" %
                                     (POOL_ROUNDS, (2 * K + 1) * S * row_bytes / 1e9),
@@ -341,12 +350,12 @@ def bench_reference(args):
     pool = [si.round_logits(ws, r, "cpu") for r in range(2)]
     K = w.k_max
     for r in range(args.warmup):
-        oracle_sample(w, [pool[r % 2][0]], [pool[r % 2][1]], n_s, 1)
+        oracle_sample(w, [pool[r % 2][0]], [pool[r % 2][1]], n_s, 1, params=variant_params(args))
     rows = 0
     t0 = time.perf_counter()
     cores = 1
     for r in range(args.steps):
-        ro, _, cores = oracle_sample(w, [pool[r % 2][0]], [pool[r % 2][1]], n_s, 1)
+        ro, _, cores = oracle_sample(w, [pool[r % 2][0]], [pool[r % 2][1]], n_s, 1, params=variant_params(args))
         rows += ro
     dt = time.perf_counter() - t0
     value = rows / dt
@@ -354,8 +363,8 @@ def bench_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt * 1e3 / max(1, args.steps), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "%s: batch %d, vocab %d, %s logits, k_max %d, %s-level %s, %d arms" %
-                               (w.name, w.n_seq, w.vocab, w.dtype, K, w.level, w.policy, w.n_arms),
+        "config": {"workload": "%s: batch %d, vocab %d, %s logits, k_max %d, %s-level %s, %d arms%s" %
+                               (w.name, w.n_seq, w.vocab, w.dtype, K, w.level, w.policy, w.n_arms, VARIANT_NOTE if args.greedy else ""),
                    "sample": "each step = one round over %d of %d sequences" % (n_s, w.n_seq)},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": "%d of %d sequences per step, %d steps" % (n_s, w.n_seq, args.steps)},
@@ -381,6 +390,7 @@ def main():
     ap.add_argument("--row-segments", type=int, default=0, help="CTAs per draft row (0 = library default)")
     ap.add_argument("--verify-cluster", type=int, default=0, help="CTAs per verify cluster (0 = library default)")
     ap.add_argument("--pool-rounds", type=int, default=POOL_ROUNDS)
+    ap.add_argument("--greedy", action="store_true", help="greedy draft + verification by matching the target's top token")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 20 if args.steps is None else args.steps

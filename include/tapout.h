@@ -108,7 +108,10 @@ typedef enum {
     TAPOUT_P_PROFILE = 32,         /* i64: 1 = time every kernel of the round with CUDA events (tapout_get_profile) */
     TAPOUT_P_VERIFY_CLUSTER = 33,  /* i64: CTAs per thread-block cluster that walks one sequence in verify: 1, 2, 4, 8
                                       (0 = chosen from vocab); reading it back gives the size in use      */
-    TAPOUT_P__COUNT = 34
+    TAPOUT_P_DRAFT_GREEDY = 34,    /* i64: 1 = the draft decodes greedily, x_i = argmax q_i (lowest index among equal maxima)
+                                      instead of a draw; features and stop rule unchanged (default 0)        */
+    TAPOUT_P_VERIFY_GREEDY = 35,   /* i64: 1 = tapout_verify accepts by matching the target's top token (see there; default 0) */
+    TAPOUT_P__COUNT = 36
 } tapout_param;
 
 /* Sticky status bits reported by tapout_get_status. */
@@ -179,6 +182,13 @@ int tapout_draft_step(tapout_t* h, const void* draft_logits, int32_t* out_token,
  *   target_logits : device, [n_seq][k_max+1][vocab] (strides TAPOUT_P_P_*)
  *   draft_tokens  : device, int32 [n_seq][k_max]; entries at positions >= n are ignored
  *   out_accept_len, out_next_token : device, int32 [n_seq]
+ * With TAPOUT_P_VERIFY_GREEDY = 1 the verification step is read literally ("accept
+ * maximal matching prefix", Algorithm 1; the target accepts the tokens "that match its
+ * predictions", Section 2): x_i is accepted iff it is the token the target ranks first
+ * at slot i (argmax_v p_i(v), lowest index among equal maxima); out_next_token is the
+ * target's own top token at the first mismatching slot, or at slot n when every token
+ * matched.  No random numbers are drawn, draft_probs is not read (it may be NULL), and a
+ * round reads |Y| + 1 target rows.
  * TAPOUT_E_BAD_STATE if no draft step ran this round or verify already ran.
  */
 int tapout_verify(tapout_t* h, const void* draft_probs, const void* target_logits,

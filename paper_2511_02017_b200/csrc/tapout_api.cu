@@ -266,11 +266,19 @@ cudaError_t launch_walk(tapout* h, const WalkArgs& a) {
                           h->cluster, h->p, h->st, h->sc, a);
 }
 
+template <int DT>
+cudaError_t launch_greedy(tapout* h, const WalkArgs& a) {
+    return launch_chained(k_verify_greedy<DT>, (unsigned)h->p.S * (unsigned)h->cluster, kThreads, 0, h->stream,
+                          h->cluster, h->p, h->st, h->sc, a);
+}
+
 int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const void* pl, int64_t p_seq, int64_t p_pos,
                 const int32_t* toks, int32_t* out_acc, int32_t* out_next) {
-    if (!h || !q || !pl || !toks || !out_acc || !out_next) return TAPOUT_E_INVALID_ARG;
+    if (!h || !pl || !toks || !out_acc || !out_next) return TAPOUT_E_INVALID_ARG;
+    const bool greedy = h->p.verify_greedy != 0;          // matching the target's top token: the draft rows are not read
+    if (!greedy && !q) return TAPOUT_E_INVALID_ARG;
     if (h->pos == 0 || h->verified) return TAPOUT_E_BAD_STATE;
-    if (!aligned16(q) || !aligned16(pl) || !stride_ok(h, q_seq) || !stride_ok(h, q_pos) || !stride_ok(h, p_seq) ||
+    if ((!greedy && !aligned16(q)) || !aligned16(pl) || !stride_ok(h, q_seq) || !stride_ok(h, q_pos) || !stride_ok(h, p_seq) ||
         !stride_ok(h, p_pos))
         return TAPOUT_E_ALIGNMENT;
     WalkArgs a = {};
@@ -280,7 +288,8 @@ int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const vo
     a.out_acc = out_acc; a.out_next = out_next;
     if (h->ev[0].size() % 2 == 1) { int rc = profile_mark(h, 0); if (rc) return rc; }
     { int rc = profile_mark(h, 1); if (rc) return rc; }
-    TP_CUDA(h, h->p.dtype == DT_BF16 ? launch_walk<DT_BF16>(h, a) : launch_walk<DT_FP32>(h, a));
+    if (greedy) TP_CUDA(h, h->p.dtype == DT_BF16 ? launch_greedy<DT_BF16>(h, a) : launch_greedy<DT_FP32>(h, a));
+    else TP_CUDA(h, h->p.dtype == DT_BF16 ? launch_walk<DT_BF16>(h, a) : launch_walk<DT_FP32>(h, a));
     TP_LAUNCHED(h);
     { int rc = profile_mark(h, 1); if (rc) return rc; }
     if (h->profile) h->prof_n[1] += 1;
@@ -343,7 +352,7 @@ int tapout_create(tapout_t** out, int n_seq, int vocab, int k_max, int n_arms, i
     p.ada_gamma = 0.2; p.ada_alpha = 0.9; p.ada_beta1 = 0.5; p.ada_beta2 = 0.9; p.ada_eps = 0.01;
     p.ada_lambda0 = 0.4; p.ada_acc0 = 1.0;
     p.reward_alpha = 0.5; p.ucb_c2 = 2.0; p.ts_mu0 = 0.0; p.ts_var0 = 1.0; p.ts_noise_var = 1.0;
-    p.ts_a0 = 1; p.ts_b0 = 1; p.reward_kind = 0; p.token_update_all = 1;
+    p.ts_a0 = 1; p.ts_b0 = 1; p.reward_kind = 0; p.token_update_all = 1; p.draft_greedy = 0; p.verify_greedy = 0;
     h->step_stride = vocab;
     h->q_seq = (int64_t)k_max * vocab; h->q_pos = vocab;
     h->p_seq = (int64_t)(k_max + 1) * vocab; h->p_pos = vocab;
@@ -424,6 +433,8 @@ int tapout_set_param_i64(tapout_t* h, int key, int64_t v) {
     case TAPOUT_P_TS_BETA_A0: if (v < 1 || v > (1 << 20)) return TAPOUT_E_INVALID_ARG; p.ts_a0 = (uint32_t)v; return TAPOUT_OK;
     case TAPOUT_P_TS_BETA_B0: if (v < 1 || v > (1 << 20)) return TAPOUT_E_INVALID_ARG; p.ts_b0 = (uint32_t)v; return TAPOUT_OK;
     case TAPOUT_P_TOKEN_UPDATE_ALL: p.token_update_all = v ? 1 : 0; return TAPOUT_OK;
+    case TAPOUT_P_DRAFT_GREEDY: p.draft_greedy = v ? 1 : 0; return TAPOUT_OK;
+    case TAPOUT_P_VERIFY_GREEDY: p.verify_greedy = v ? 1 : 0; return TAPOUT_OK;
     case TAPOUT_P_TOKEN_OUT_STRIDE: if (v < 1) return TAPOUT_E_INVALID_ARG; h->tok_stride = v; return TAPOUT_OK;
     case TAPOUT_P_PROFILE: h->profile = v != 0; return TAPOUT_OK;
     case TAPOUT_P_ROW_SEGMENTS: {
@@ -491,6 +502,8 @@ int tapout_get_param_i64(const tapout_t* h, int key, int64_t* v) {
     case TAPOUT_P_TS_BETA_A0: *v = p.ts_a0; return TAPOUT_OK;
     case TAPOUT_P_TS_BETA_B0: *v = p.ts_b0; return TAPOUT_OK;
     case TAPOUT_P_TOKEN_UPDATE_ALL: *v = p.token_update_all; return TAPOUT_OK;
+    case TAPOUT_P_DRAFT_GREEDY: *v = p.draft_greedy; return TAPOUT_OK;
+    case TAPOUT_P_VERIFY_GREEDY: *v = p.verify_greedy; return TAPOUT_OK;
     case TAPOUT_P_ROW_SEGMENTS: *v = p.nseg; return TAPOUT_OK;
     case TAPOUT_P_VERIFY_CLUSTER: *v = h->cluster; return TAPOUT_OK;
     case TAPOUT_P_TOKEN_OUT_STRIDE: *v = h->tok_stride; return TAPOUT_OK;

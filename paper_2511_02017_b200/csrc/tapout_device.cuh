@@ -37,6 +37,7 @@ struct Params {
     double reward_alpha, ucb_c2, ts_mu0, ts_var0, ts_noise_var;
     uint32_t ts_a0, ts_b0;
     int reward_kind, token_update_all;
+    int draft_greedy, verify_greedy;     // greedy decoding of the draft; verification by matching the target's top token
     int nseg, NC;                        // CTAs per draft row, chunks per row
 };
 
@@ -216,6 +217,33 @@ template <> __device__ __forceinline__ float lane_max<DT_FP32>(const uint4 (&v)[
     for (int j = 0; j < kVecPerLane; ++j) {
         m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(v[j].x), __uint_as_float(v[j].y)),
                            fmaxf(__uint_as_float(v[j].z), __uint_as_float(v[j].w))));
+    }
+    return m;
+}
+
+// Largest element of the lane's 4 vectors with NaN kept: the result is NaN as soon as one entry is (the pass
+// that only looks for the maximum has no sums for a NaN to surface in).
+template <int DT> __device__ __forceinline__ float lane_max_nan(const uint4 (&v)[kVecPerLane]);
+template <> __device__ __forceinline__ float lane_max_nan<DT_BF16>(const uint4 (&v)[kVecPerLane]) {
+    __nv_bfloat162 q[kVecPerLane];
+#pragma unroll
+    for (int j = 0; j < kVecPerLane; ++j)
+        q[j] = __hmax2_nan(__hmax2_nan(as_bf162(v[j].x), as_bf162(v[j].y)), __hmax2_nan(as_bf162(v[j].z), as_bf162(v[j].w)));
+    const uint32_t b = as_u32(__hmax2_nan(__hmax2_nan(q[0], q[1]), __hmax2_nan(q[2], q[3])));
+    const float lo = __uint_as_float(b << 16), hi = __uint_as_float(b & 0xffff0000u);
+    float r;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+template <> __device__ __forceinline__ float lane_max_nan<DT_FP32>(const uint4 (&v)[kVecPerLane]) {
+    float m = neg_inf();
+#pragma unroll
+    for (int j = 0; j < kVecPerLane; ++j) {
+        float a, b;
+        asm("max.NaN.f32 %0, %1, %2;" : "=f"(a) : "f"(__uint_as_float(v[j].x)), "f"(__uint_as_float(v[j].y)));
+        asm("max.NaN.f32 %0, %1, %2;" : "=f"(b) : "f"(__uint_as_float(v[j].z)), "f"(__uint_as_float(v[j].w)));
+        asm("max.NaN.f32 %0, %1, %2;" : "=f"(a) : "f"(a), "f"(b));
+        asm("max.NaN.f32 %0, %1, %2;" : "=f"(m) : "f"(m), "f"(a));
     }
     return m;
 }

@@ -95,6 +95,7 @@ __device__ __forceinline__ void store_segrec(SegRec* g, const SegRec& r) {
 template <int DT, bool FEATURES, int ROLE>
 __device__ __forceinline__ void finish_row(const Params& p, const State& st, const Scratch& sc, const StepArgs& a, int s,
                                            int n_warps_stream, int lane) {
+    if (!FEATURES && ROLE == 2 && p.draft_greedy) return;        // greedy decoding: the token is the argmax role 1 finds
     const char* row = reinterpret_cast<const char*>(a.logits) + (size_t)s * a.row_stride * Elem<DT>::BYTES;
     const float2* part = sc.cdf + (size_t)s * p.NC;
     const float c = a.c;
@@ -248,6 +249,7 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
         fo[0] = (float)m_s; fo[1] = (float)lse; fo[2] = (float)p1; fo[3] = (float)p2; fo[4] = (float)H;
         fo[5] = (float)first;
         st.lse_q[(size_t)s * p.K + pos] = lse;
+        if (p.draft_greedy) a.out_token[(size_t)s * a.tok_stride] = first;
         int rule = 0;                        // a select chain: indexing the parameter array would move it to local memory
 #pragma unroll
         for (int k = 0; k < kMaxArms; ++k) rule = (k == arm) ? p.rule_of_arm[k] : rule;
@@ -265,7 +267,7 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
             sc.list[(size_t)nslot * p.S + atomicAdd(&sc.count[nslot], 1)] = s;
         }
     }
-    if (ROLE == 0) {
+    if (ROLE == 0 && !p.draft_greedy) {
         // x_i ~ softmax(row) inside the chunk, from the weights the streaming pass summed
         int tok = -1;
         if (chunk >= 0) tok = pick_softmax_block<DT>(vx, p.V, chunk, c, kch, rem * draw_scale, lane);
@@ -652,6 +654,100 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
             if (acc_len < n) atomicAdd(&sc.status[3], 1ull);
         }
         if (mine && !bad) a.out_next[s] = next;
+    }
+}
+
+// ============================================================================================
+// Verification read literally (Algorithm 1: "accept maximal matching prefix"): x_i is accepted iff it is
+// the token the target ranks first at slot i, and the final token is the target's top token at the first
+// mismatch (or at slot n).  Same layout as the sampling walk -- one cluster per sequence, longest drafts
+// first, CTA r streams the r-th slice of each target row -- but the pass only looks for the row maximum:
+// every warp keeps (largest value, lowest chunk of its own that holds it), the cluster exchanges the
+// records through distributed shared memory, and warp 0 of every CTA re-reads the one winning chunk
+// (L2) for the token index.  Rows after the first mismatch are not read.
+// ============================================================================================
+struct GreedyShared {
+    float2 gather[2][kMaxCluster][kWarps];   // per warp (maximum or NaN, its lowest chunk as int bits), by row parity
+    int dec[2], top[2];                      // decision of the row (1 match, 0 mismatch / last row, -1 unusable row), top token
+};
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, kWalkResident)
+k_verify_greedy(Params p, State st, Scratch sc, WalkArgs a)
+{
+    constexpr int ESZ = Elem<DT>::BYTES;
+    __shared__ GreedyShared sh;
+    cg::cluster_group cl = cg::this_cluster();
+    const int CS = (int)cl.num_blocks();
+    const int rank = (int)cl.block_rank();
+    const int cid = blockIdx.x / CS;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    pdl_wait();                                           // before the trigger: see k_verify_walk
+    pdl_trigger();
+    const long long e = sc.stopped[p.S - 1 - cid];
+    const int n_act = sc.count[a.slot];
+    int s = (int)(unsigned)e, n = (int)(e >> 32);
+    if (cid < n_act) { s = sc.list[(size_t)a.slot * p.S + cid]; n = a.pos; }
+    const char* pbase = reinterpret_cast<const char*>(a.plog) + (size_t)s * a.p_seq * ESZ;
+    const int c0 = (int)(((long long)rank * p.NC) / CS);
+    const int c1 = (int)(((long long)(rank + 1) * p.NC) / CS);
+
+    int acc_len = n, next = -1;
+    bool bad = false;
+    int x_next = (warp == 0 && n > 0) ? a.toks[(size_t)s * p.K] : -1;
+    for (int i = 0; i <= n; ++i) {
+        const char* prow = pbase + (size_t)i * a.p_pos * ESZ;
+        const int par = i & 1;
+        const int x = x_next;                             // asked for a row ahead: it is here by the time it is compared
+        if (warp == 0 && i + 1 < n) x_next = a.toks[(size_t)s * p.K + i + 1];
+        float ref = neg_inf();
+        int best = 0x7fffffff;
+        bool nan = false;
+        for (int ch = c0 + warp; ch < c1; ch += kWarps) {
+            uint4 v[kVecPerLane];
+            load_chunk<DT>(prow, p.V, ch, lane, v);
+            const float lm = lane_max_nan<DT>(v);
+            nan = nan || (lm != lm);
+            const float M = warp_max_redux(lm);           // NaN lanes are skipped here and reported below
+            if (M > ref) { ref = M; best = ch; }
+        }
+        if (__any_sync(0xffffffffu, nan)) ref = __int_as_float(0x7fc00000);
+        if (lane < CS) cl.map_shared_rank(&sh, lane)->gather[par][rank][warp] = make_float2(ref, __int_as_float(best));
+        cl.sync();
+        if (warp == 0) {
+            const int nrec = CS * kWarps;                 // <= 64: two records per lane
+            const float2* g = &sh.gather[par][0][0];
+            float2 r0 = make_float2(neg_inf(), __int_as_float(0x7fffffff)), r1 = r0;
+            if (lane < nrec) r0 = g[lane];
+            if (lane + 32 < nrec) r1 = g[lane + 32];
+            const bool any_nan = __any_sync(0xffffffffu, r0.x != r0.x || r1.x != r1.x);
+            const float m = warp_max_f(fmaxf(r0.x, r1.x));
+            int dec = -1, top = -1;
+            if (!any_nan && m > neg_inf() && m < CUDART_INF_F) {
+                int chunk = 0x7fffffff;
+                if (r0.x == m) chunk = __float_as_int(r0.y);
+                if (r1.x == m) chunk = min(chunk, __float_as_int(r1.y));
+                chunk = __reduce_min_sync(0xffffffffu, chunk);
+                uint4 vt[4];
+                load_lane_block<DT>(prow, p.V, chunk, lane, vt);
+                int cnt;
+                float below;
+                scan_top_block<DT>(vt, p.V, chunk, m, lane, cnt, top, below);
+                dec = (i < n && x == top) ? 1 : 0;
+            }
+            if (lane == 0) { sh.dec[par] = dec; sh.top[par] = top; }
+        }
+        __syncthreads();                     // the slots of this parity are rewritten two rows on, behind a cluster barrier
+        const int dec = sh.dec[par];
+        if (dec != 1) { acc_len = i; next = sh.top[par]; bad = dec < 0; break; }
+    }
+    if (tid == 0 && rank == 0) {
+        if (bad) atomicOr(&sc.status[0], 2ull);
+        st.accept_len[s] = acc_len;
+        a.out_acc[s] = acc_len;
+        a.out_next[s] = bad ? -1 : next;
+        atomicAdd(&sc.status[2], (unsigned long long)(acc_len + 1));
     }
 }
 

@@ -1,0 +1,141 @@
+"""GPU parity of the greedy variant (draft token = argmax q_i; verification by matching the target's top
+token) against the oracle.  Everything here is integer work: tokens, accepted lengths and final tokens must
+be equal outright, so the lockstep report may show flips for the continue mask only."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2511_02017_b200 import binding as tp
+from paper_2511_02017_b200 import synth_inputs as si
+from tests.lockstep import make_device, run_lockstep
+from tests.test_gpu_parity import peaked_logits
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+GREEDY = dict(draft_greedy=1, verify_greedy=1)
+
+
+def _assert_exact(rep):
+    assert rep.ok(), "\n".join(rep.failures[:10]) + "\n" + rep.summary()
+    assert rep.flips["token"] == rep.flips["accept"] == rep.flips["next"] == 0, rep.summary()
+    print(rep.summary())
+
+
+def half_peaked_logits(w, rnd, device):
+    """peaked_logits for the even sequences (draft and target then mostly agree on the top token), the plain
+    generator for the odd ones (they mostly disagree): matched prefixes of every length."""
+    d0, t0 = si.round_logits(w, rnd, device)
+    d1, t1 = peaked_logits(w, rnd, device)
+    d0[::2], t0[::2] = d1[::2], t1[::2]
+    return d0, t0
+
+
+@pytest.mark.parametrize("name,S,rounds", [("batch64", 10, 5), ("batch256_ts", 8, 5), ("throughput", 12, 5), ("shift", 5, 3)])
+def test_greedy_lockstep_full_vocab(name, S, rounds):
+    w = si.scaled(si.WORKLOADS[name], n_seq=S)
+    rep, dev, _ = run_lockstep(w, rounds, device=DEV, logits_fn=half_peaked_logits, dev_params=GREEDY, orc_params=GREEDY)
+    _assert_exact(rep)
+    assert rep.rows_dev == rep.rows_oracle              # a + 1 target rows per sequence, no residual rows
+    assert 0.3 < rep.mean_accepted
+    dev.destroy()
+
+
+@pytest.mark.parametrize("dtype,vocab", [("bf16", 20008), ("fp32", 5001 * 4), ("bf16", 1032), ("fp32", 520)])
+@pytest.mark.parametrize("policy,level", [("ucb1", "seq"), ("ts", "token")])
+def test_greedy_lockstep_many_rounds(dtype, vocab, policy, level):
+    w = si.Workload("gr", 9, vocab, dtype, 6, 1, 5, policy, level, seed=81, sigma="per_seq:0.2:1.5")
+    rep, dev, _ = run_lockstep(w, 30, device=DEV, logits_fn=half_peaked_logits, dev_params=GREEDY, orc_params=GREEDY)
+    _assert_exact(rep)
+    dev.destroy()
+
+
+@pytest.mark.parametrize("combo", [dict(draft_greedy=1), dict(verify_greedy=1)])
+def test_each_switch_alone(combo):
+    """Greedy draft under speculative-sampling verification, and sampled drafts under greedy verification."""
+    w = si.Workload("gr1", 8, 4104, "bf16", 5, 1, 5, "ucb1", "seq", seed=82)
+    rep, dev, _ = run_lockstep(w, 16, device=DEV, logits_fn=peaked_logits, dev_params=combo, orc_params=combo)
+    assert rep.ok(), "\n".join(rep.failures[:10]) + "\n" + rep.summary()
+    dev.destroy()
+
+
+def test_equal_maxima_across_chunks_and_cluster_slices_and_unusable_rows():
+    """The top token is the lowest index among equal maxima wherever the copies sit (same chunk, other chunk,
+    another CTA's slice of the row); rows behind the first mismatch are never read; a NaN, a row without a
+    finite entry or an infinite maximum in a needed row ends the walk with token -1."""
+    S, V, K = 12, 20008, 5
+    w = si.Workload("ties", S, V, "bf16", K, 1, 1, "ucb1", "seq", seed=83)
+    spots = [(3, 4), (3, 700), (3, 1100), (500, 19999), (9000, 11000), (1023, 1024), (20006, 20007), (0, 20007)]
+
+    def gen(w_, rnd, device):
+        d, t = si.round_logits(w_, rnd, device)
+        for s in range(S):
+            lo, hi = spots[(s + rnd) % len(spots)]
+            for i in range(K + 1):
+                t[s, i, lo] = t[s, i, hi] = 40.0
+            for i in range(K):
+                d[s, i, hi if (s + i) % 4 == 3 else lo] = 40.0          # the draft picks the higher copy now and then
+        t[1, 3:] = float("nan")             # behind sequence 1's first mismatch (slot 2: (1 + 2) % 4 == 3)
+        t[2, 0, 77] = float("nan")          # a needed row
+        t[4, 1, :] = float("-inf")
+        t[5, 0, 9] = float("inf")
+        return d, t
+    arms = [tp.RULE_STATIC]
+    params = dict(arms=arms, **GREEDY)
+    rep, dev, ora = run_lockstep(w, 4, device=DEV, logits_fn=gen, dev_params=params, orc_params=params)
+    _assert_exact(rep)
+    assert dev.get_status()["bits"] == tp.ST_BAD_TARGET_ROW == ora.status
+    dev.destroy()
+
+
+def test_greedy_verify_ignores_the_draft_tensor_and_any_token_value():
+    S, V, K = 3, 2056, 3
+    t = tp.Tapout(S, V, K, 1, tp.POLICY_UCB1, tp.LEVEL_SEQ, arms=[tp.RULE_STATIC], step_row_stride=K * V, **GREEDY)
+    g = torch.Generator(device="cpu")
+    g.manual_seed(5)
+    p = (torch.randn((S, K + 1, V), generator=g) * 3).to(torch.bfloat16).to(DEV)
+    d = p[:, :K].contiguous()
+    tok = torch.empty(S, dtype=torch.int32, device=DEV)
+    cont = torch.empty(S, dtype=torch.uint8, device=DEV)
+    toks = torch.zeros((S, K), dtype=torch.int32, device=DEV)
+    for i in range(K):
+        t.draft_step(d[:, i, :], tok, cont)
+        toks[:, i] = tok
+    top = p.float().argmax(dim=2).to(torch.int32)
+    assert torch.equal(toks, top[:, :K])                 # identical models: the draft's argmax is the target's
+    toks[1, 1] = V + 5                                   # outside the vocabulary: simply not the target's token
+    toks[2, 0] = -3
+    acc = torch.empty(S, dtype=torch.int32, device=DEV)
+    nxt = torch.empty(S, dtype=torch.int32, device=DEV)
+    t.verify(None, p, toks, acc, nxt)
+    assert acc.cpu().tolist() == [K, 1, 0]
+    assert nxt.cpu().tolist() == [int(top[0, K]), int(top[1, 1]), int(top[2, 0])]
+    assert t.get_status()["bits"] == 0
+    t.update()
+    t.destroy()
+
+
+def test_greedy_full_size_round_call_against_separate_calls_and_oracle_sample():
+    """The bench workload at full size: tapout_round with both switches against the separate calls (all
+    sequences, bitwise), and the separate calls against the oracle on a sample of sequences."""
+    w = si.WORKLOADS["throughput"]
+    S, K = w.n_seq, w.k_max
+    sample = sorted(np.random.default_rng(12).choice(S, size=5, replace=False).tolist())
+    rep, a, _ = run_lockstep(w, 3, sample=sample, device=DEV, dev_params=dict(token_out_stride=1, **GREEDY), orc_params=GREEDY)
+    _assert_exact(rep)
+    b = make_device(w, token_out_stride=K, **GREEDY)
+    toks_b = torch.empty((S, K), dtype=torch.int32, device=DEV)
+    cont_b = torch.empty(S, dtype=torch.uint8, device=DEV)
+    acc_b = torch.empty(S, dtype=torch.int32, device=DEV)
+    nxt_b = torch.empty(S, dtype=torch.int32, device=DEV)
+    for rnd in range(3):
+        d, t = si.round_logits(w, rnd, DEV)
+        b.round(d, t, toks_b, cont_b, acc_b, nxt_b)
+        del d, t
+    torch.cuda.synchronize()
+    sa, sb = a.get_state(), b.get_state()
+    for name in ("cnt", "rsum", "lambda", "acc_rate", "reward", "accept_len", "n_drafted"):
+        assert np.array_equal(sa[name], sb[name]), name
+    assert a.get_status() == b.get_status()
+    a.destroy()
+    b.destroy()
+    torch.cuda.empty_cache()
