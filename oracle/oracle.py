@@ -68,6 +68,8 @@ def lib():
         L.orc_ts_beta_select.argtypes = [vp, vp, i32, u32, u32, u64, u32, u32, u32, vp]
         L.orc_verify_sequence.argtypes = [vp, C.c_long, vp, C.c_long, i32, i32, C.c_float, C.c_float,
                                           vp, i32, vp, u64, u32, u32, dbl, vp, C.POINTER(VerifyOut)]
+        L.orc_verify_sequence_qprobs.argtypes = [vp, C.c_long, vp, C.c_long, i32, i32, C.c_float, vp, i32, u64, u32, u32,
+                                                 dbl, vp, C.POINTER(VerifyOut)]
         L.orc_verify_sequence_greedy.argtypes = [vp, C.c_long, i32, i32, C.c_float, vp, i32, C.POINTER(VerifyOut)]
         L.orc_create.restype = vp
         L.orc_create.argtypes = [i32] * 6
@@ -213,6 +215,19 @@ def verify_sequence(q_rows, p_rows, x, lse_q, seed, seq, rnd, inv_Tq=1.0, inv_Tp
     lib().orc_verify_sequence(_ptr(q_rows), V, _ptr(p_rows), V, _dtype_code(p_rows), V,
                               np.float32(inv_Tq), np.float32(inv_Tp), _ptr(x), x.shape[0], _ptr(lse_q),
                               seed, seq, rnd, tol, _ptr(scratch), C.byref(out))
+    return out
+
+
+def verify_sequence_qprobs(q_probs, p_rows, x, seed, seq, rnd, inv_Tp=1.0, tol=1e-6):
+    """q_probs [>= n][V] float32 probabilities, p_rows [>= n+1][V] logits, x [n] tokens."""
+    q_probs = np.ascontiguousarray(q_probs, dtype=np.float32)
+    p_rows = np.ascontiguousarray(p_rows)
+    x = np.ascontiguousarray(x, dtype=np.int32)
+    V = p_rows.shape[1]
+    scratch = np.zeros(2 * V)
+    out = VerifyOut()
+    lib().orc_verify_sequence_qprobs(_ptr(q_probs), V, _ptr(p_rows), V, _dtype_code(p_rows), V, np.float32(inv_Tp),
+                                     _ptr(x), x.shape[0], seed, seq, rnd, tol, _ptr(scratch), C.byref(out))
     return out
 
 

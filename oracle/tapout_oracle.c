@@ -453,6 +453,59 @@ void orc_verify_sequence(const void* q_rows, long q_pos_stride, const void* p_ro
     }
 }
 
+/* The same walk when the caller hands the draft distributions over as
+ * normalised fp32 probabilities instead of logits: q_i(v) is the stored number
+ * itself.  ratio = p_i(x_i) / q_i(x_i) in IEEE arithmetic (q = 0 < p accepts,
+ * 0/0 is NaN and rejects); the residual is max(0, p - q) with the same q.
+ * q_rows: n rows of V floats, q_pos_stride floats apart.  scratch: 2*V doubles. */
+void orc_verify_sequence_qprobs(const float* q_rows, long q_pos_stride, const void* p_rows, long p_pos_stride,
+                                int dtype, int V, float inv_Tp, const int32_t* x, int n,
+                                uint64_t seed, uint32_t seq, uint32_t round, double tol,
+                                double* scratch, orc_verify_out* out)
+{
+    size_t esz = (dtype == ORC_FP32) ? 4 : 2;
+    double* wp = scratch;
+    double* res = scratch + V;
+    memset(out, 0, sizeof *out);
+    out->next_token = -1; out->next_lo = -1; out->next_hi = -1;
+
+    int a = n;
+    orc_rowstats sp;
+    for (int i = 0; i < n; ++i) {
+        const void* prow = (const char*)p_rows + (size_t)i * p_pos_stride * esz;
+        if (!orc_row_stats(prow, dtype, V, inv_Tp, wp, &sp)) { out->bad_target = 1; a = i; out->accept_len = a; return; }
+        double px = exp(load_logit(prow, dtype, x[i]) * (double)inv_Tp - sp.lse);
+        double qx = (double)q_rows[(size_t)i * q_pos_stride + x[i]];
+        double ratio = px / qx;
+        double u = orc_rng_uniform(seed, seq, round, (uint32_t)i, ORC_RNG_ACCEPT, 0, 0, 0);
+        out->ratio_at_stop = ratio;
+        if (fabs(u - ratio) <= tol) out->near_accept = 1;
+        if (!(u < ratio)) { a = i; break; }
+    }
+    out->accept_len = a;
+
+    double u2 = orc_rng_uniform(seed, seq, round, (uint32_t)a, ORC_RNG_RESAMPLE, 0, 0, 0);
+    const void* prow = (const char*)p_rows + (size_t)a * p_pos_stride * esz;
+    if (a == n) {
+        if (!orc_row_stats(prow, dtype, V, inv_Tp, wp, &sp)) { out->bad_target = 1; return; }
+        out->next_token = orc_sample_cdf(wp, V, sp.W, u2, tol, &out->next_lo, &out->next_hi);
+        return;
+    }
+    const float* qrow = q_rows + (size_t)a * q_pos_stride;
+    double Z = 0.0;
+    for (int v = 0; v < V; ++v) {
+        double r = wp[v] / sp.W - (double)qrow[v];
+        res[v] = r > 0.0 ? r : 0.0;
+        Z += res[v];
+    }
+    if (Z > 0.0) {
+        out->next_token = orc_sample_cdf(res, V, Z, u2, tol, &out->next_lo, &out->next_hi);
+    } else {
+        out->zero_residual = 1;
+        out->next_token = orc_sample_cdf(wp, V, sp.W, u2, tol, &out->next_lo, &out->next_hi);
+    }
+}
+
 /* ------------------------------------------------------------------------- */
 /* Verification read literally (Algorithm 1: "accept maximal matching prefix"; */
 /* Section 2: the target accepts the drafted tokens "that match its           */
@@ -502,6 +555,7 @@ typedef struct {
     int token_update_all;        /* 1: every drafted position gets r_i = [i <= a]; 0: only i <= a+1 */
     int draft_greedy;            /* 1: x_i = argmax q_i instead of a draw                        */
     int verify_greedy;           /* 1: verification by matching the target's argmax (see above)  */
+    int q_format;                /* verify's draft tensor: 0 = logits, 1 = normalised fp32 probabilities */
     double tol;                  /* near-threshold band, 1e-6 */
     /* per-sequence global ids (RNG stream of local sequence s is seq_id[s]) */
     uint32_t* seq_id;
@@ -697,6 +751,11 @@ int orc_verify(orc_t* h, const void* draft_logits, long q_seq_stride, long q_pos
         if (h->verify_greedy)
             orc_verify_sequence_greedy((const char*)target_logits + (size_t)s * p_seq_stride * esz, p_pos_stride,
                                        h->dtype, h->V, h->inv_Tp, draft_tokens + (size_t)s * h->K, n, &vo);
+        else if (h->q_format == 1)
+            orc_verify_sequence_qprobs((const float*)draft_logits + (size_t)s * q_seq_stride, q_pos_stride,
+                                       (const char*)target_logits + (size_t)s * p_seq_stride * esz, p_pos_stride,
+                                       h->dtype, h->V, h->inv_Tp, draft_tokens + (size_t)s * h->K, n,
+                                       h->seed, h->seq_id[s], h->round, h->tol, scratch, &vo);
         else
             orc_verify_sequence((const char*)draft_logits + (size_t)s * q_seq_stride * esz, q_pos_stride,
                                 (const char*)target_logits + (size_t)s * p_seq_stride * esz, p_pos_stride,
@@ -792,6 +851,7 @@ int orc_set_param(orc_t* h, const char* key, double v)
     else if (K_("token_update_all")) h->token_update_all = (int)v;
     else if (K_("draft_greedy")) h->draft_greedy = (int)v;
     else if (K_("verify_greedy")) h->verify_greedy = (int)v;
+    else if (K_("q_format")) h->q_format = (int)v;
     else if (K_("tol")) h->tol = v;
     else return -1;
 #undef K_

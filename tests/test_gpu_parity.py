@@ -218,6 +218,19 @@ def test_lockstep_full_size_sampled_sequences(name, rounds, n_sample):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("policy", ["ts", "ucb1"])
+def test_token_level_bandits_at_the_papers_draft_cap(policy):
+    """gamma = 128, the cap the paper runs with: 128 bandits per sequence at token level, a fixed-length arm in
+    the pool so that drafts reach far positions, and Beta draws that grow with the play counts."""
+    arms = [tp.RULE_STATIC, tp.RULE_SVIP, tp.RULE_STATIC, tp.RULE_MARGIN, tp.RULE_STATIC]
+    w = si.Workload("k128", 5, 2056, "bf16", 128, 1, 5, policy, "token", seed=72)
+    rep, dev, _ = run_lockstep(w, 8, device=DEV, logits_fn=peaked_logits, dev_params=dict(arms=arms),
+                               orc_params=dict(arms=arms), check_state_every=4)
+    _assert_clean(rep)
+    assert rep.mean_drafted > 2
+    dev.destroy()
+
+
 @pytest.mark.parametrize("dtype,vocab", [("bf16", 300008), ("fp32", 140004)])
 def test_vocabulary_beyond_the_register_resident_chunk_table(dtype, vocab):
     """More than 256 chunks per row: the finish kernel searches the chunk partials in memory instead of registers."""
