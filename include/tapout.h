@@ -111,8 +111,15 @@ typedef enum {
     TAPOUT_P_DRAFT_GREEDY = 34,    /* i64: 1 = the draft decodes greedily, x_i = argmax q_i (lowest index among equal maxima)
                                       instead of a draw; features and stop rule unchanged (default 0)        */
     TAPOUT_P_VERIFY_GREEDY = 35,   /* i64: 1 = tapout_verify accepts by matching the target's top token (see there; default 0) */
-    TAPOUT_P__COUNT = 36
+    TAPOUT_P_Q_FORMAT = 36,        /* i64: what tapout_verify's draft_probs holds: TAPOUT_Q_LOGITS (default) or TAPOUT_Q_PROBS_F32 */
+    TAPOUT_P__COUNT = 37
 } tapout_param;
+
+/* Values of TAPOUT_P_Q_FORMAT. */
+enum {
+    TAPOUT_Q_LOGITS = 0,       /* the draft logits tensor the rows of which went through tapout_draft_step (fast path)  */
+    TAPOUT_Q_PROBS_F32 = 1     /* normalised probabilities, float32 [n_seq][k_max][vocab]; strides TAPOUT_P_Q_* in floats */
+};
 
 /* Sticky status bits reported by tapout_get_status. */
 #define TAPOUT_ST_BAD_DRAFT_ROW 1ull   /* a draft row was unusable                              */
@@ -182,6 +189,12 @@ int tapout_draft_step(tapout_t* h, const void* draft_logits, int32_t* out_token,
  *   target_logits : device, [n_seq][k_max+1][vocab] (strides TAPOUT_P_P_*)
  *   draft_tokens  : device, int32 [n_seq][k_max]; entries at positions >= n are ignored
  *   out_accept_len, out_next_token : device, int32 [n_seq]
+ * With TAPOUT_P_Q_FORMAT = TAPOUT_Q_PROBS_F32 draft_probs holds the draft distributions
+ * themselves (float32, normalised by the caller, 16-byte aligned rows): q_i(v) is the
+ * stored number, the ratio is p_i(x_i) / q_i(x_i) in IEEE arithmetic (q = 0 < p accepts,
+ * 0 / 0 rejects) and the residual is max(0, p - q) with the same q.  A slower path (rows
+ * twice as wide as bf16 logits); tapout_round and tapout_round_host, which take one draft
+ * tensor for both uses, return TAPOUT_E_UNSUPPORTED in this format.
  * With TAPOUT_P_VERIFY_GREEDY = 1 the verification step is read literally ("accept
  * maximal matching prefix", Algorithm 1; the target accepts the tokens "that match its
  * predictions", Section 2): x_i is accepted iff it is the token the target ranks first

@@ -17,6 +17,7 @@ STATIC_MAX_ROWS, STATIC_MAX_VOCAB = 64, 262144
 POLICY_UCB1, POLICY_TS, POLICY_UCB_TUNED = 0, 1, 2
 LEVEL_SEQ, LEVEL_TOKEN = 0, 1
 DTYPE_FP32, DTYPE_BF16 = 0, 1
+Q_LOGITS, Q_PROBS_F32 = 0, 1
 RULE_MAXCONF, RULE_SVIP, RULE_ADAEDL, RULE_SVIPDIFF, RULE_MARGIN, RULE_STATIC = range(6)
 ST_BAD_DRAFT_ROW, ST_BAD_TARGET_ROW, ST_ZERO_RESIDUAL, ST_BAD_TOKEN = 1, 2, 4, 8
 
@@ -26,12 +27,12 @@ _PARAM_NAMES = [
     "q_pos_stride", "p_seq_stride", "p_pos_stride", "h_maxconf", "h_svip", "h_diff", "h_margin", "ada_gamma",
     "ada_alpha", "ada_beta1", "ada_beta2", "ada_eps", "ada_lambda0", "ada_acc0", "reward_alpha", "reward_kind",
     "ucb_c2", "ts_mu0", "ts_var0", "ts_noise_var", "ts_beta_a0", "ts_beta_b0", "token_update_all", "row_segments",
-    "token_out_stride", "profile", "verify_cluster", "draft_greedy", "verify_greedy",
+    "token_out_stride", "profile", "verify_cluster", "draft_greedy", "verify_greedy", "q_format",
 ]
 PARAM = {n: i for i, n in enumerate(_PARAM_NAMES)}
 _INT_PARAMS = {"seed", "dtype", "seq_offset", "step_row_stride", "q_seq_stride", "q_pos_stride", "p_seq_stride",
                "p_pos_stride", "reward_kind", "ts_beta_a0", "ts_beta_b0", "token_update_all", "row_segments",
-               "token_out_stride", "profile", "verify_cluster", "draft_greedy", "verify_greedy"}
+               "token_out_stride", "profile", "verify_cluster", "draft_greedy", "verify_greedy", "q_format"}
 
 EXPORTS = [
     "tapout_strerror", "tapout_last_cuda_error", "tapout_create", "tapout_destroy", "tapout_set_stream",

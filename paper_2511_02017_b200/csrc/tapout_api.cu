@@ -47,6 +47,7 @@ struct tapout {
     int grid_rows = 0;
     int cluster_user = 0, cluster = 1;   // CTAs per verify cluster: requested (0 = automatic) and in use
     size_t walk_smem = 0;
+    bool q_probs = false;                // tapout_verify's draft tensor holds fp32 probabilities, not logits
     bool arms_ready = false;             // the arms of round `round` are chosen and the round's lists are set up
     // host-round staging
     char* d_stage = nullptr;
@@ -131,14 +132,16 @@ int setup_scratch(tapout* h) {
     for (;; cs >>= 1) {
         h->walk_smem = sizeof(float2) * (size_t)((p.NC + cs - 1) / cs + 1);
         if (h->walk_smem > 160 * 1024) return TAPOUT_E_UNSUPPORTED;      // vocabulary too large for the chunk table
-        const int fit = (p.dtype == DT_BF16) ? cluster_fits(h, k_verify_walk<DT_BF16>, cs, h->walk_smem)
-                                             : cluster_fits(h, k_verify_walk<DT_FP32>, cs, h->walk_smem);
+        const int fit = (p.dtype == DT_BF16) ? cluster_fits(h, (k_verify_walk<DT_BF16, false>), cs, h->walk_smem)
+                                             : cluster_fits(h, (k_verify_walk<DT_FP32, false>), cs, h->walk_smem);
         if (fit > 0 || cs == 1) break;
     }
     h->cluster = cs;
     if (h->walk_smem > 40 * 1024) {
-        TP_CUDA(h, cudaFuncSetAttribute(k_verify_walk<DT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
-        TP_CUDA(h, cudaFuncSetAttribute(k_verify_walk<DT_FP32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
+        TP_CUDA(h, cudaFuncSetAttribute((k_verify_walk<DT_BF16, false>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
+        TP_CUDA(h, cudaFuncSetAttribute((k_verify_walk<DT_FP32, false>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
+        TP_CUDA(h, cudaFuncSetAttribute((k_verify_walk<DT_BF16, true>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
+        TP_CUDA(h, cudaFuncSetAttribute((k_verify_walk<DT_FP32, true>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
     }
 
     if (h->d_scratch) { cudaFree(h->d_scratch); h->d_scratch = nullptr; }
@@ -260,9 +263,9 @@ int draft_step_impl(tapout* h, const void* logits, int64_t stride, int32_t* out_
     return TAPOUT_OK;
 }
 
-template <int DT>
+template <int DT, bool QP>
 cudaError_t launch_walk(tapout* h, const WalkArgs& a) {
-    return launch_chained(k_verify_walk<DT>, (unsigned)h->p.S * (unsigned)h->cluster, kThreads, h->walk_smem, h->stream,
+    return launch_chained(k_verify_walk<DT, QP>, (unsigned)h->p.S * (unsigned)h->cluster, kThreads, h->walk_smem, h->stream,
                           h->cluster, h->p, h->st, h->sc, a);
 }
 
@@ -278,8 +281,9 @@ int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const vo
     const bool greedy = h->p.verify_greedy != 0;          // matching the target's top token: the draft rows are not read
     if (!greedy && !q) return TAPOUT_E_INVALID_ARG;
     if (h->pos == 0 || h->verified) return TAPOUT_E_BAD_STATE;
-    if ((!greedy && !aligned16(q)) || !aligned16(pl) || !stride_ok(h, q_seq) || !stride_ok(h, q_pos) || !stride_ok(h, p_seq) ||
-        !stride_ok(h, p_pos))
+    const bool q_ok = h->q_probs ? (q_seq > 0 && q_pos > 0 && q_seq % 4 == 0 && q_pos % 4 == 0)      // fp32 rows
+                                 : (stride_ok(h, q_seq) && stride_ok(h, q_pos));
+    if ((!greedy && (!aligned16(q) || !q_ok)) || !aligned16(pl) || !stride_ok(h, p_seq) || !stride_ok(h, p_pos))
         return TAPOUT_E_ALIGNMENT;
     WalkArgs a = {};
     a.qlog = q; a.q_seq = q_seq; a.q_pos = q_pos; a.plog = pl; a.p_seq = p_seq; a.p_pos = p_pos;
@@ -288,8 +292,12 @@ int verify_impl(tapout* h, const void* q, int64_t q_seq, int64_t q_pos, const vo
     a.out_acc = out_acc; a.out_next = out_next;
     if (h->ev[0].size() % 2 == 1) { int rc = profile_mark(h, 0); if (rc) return rc; }
     { int rc = profile_mark(h, 1); if (rc) return rc; }
-    if (greedy) TP_CUDA(h, h->p.dtype == DT_BF16 ? launch_greedy<DT_BF16>(h, a) : launch_greedy<DT_FP32>(h, a));
-    else TP_CUDA(h, h->p.dtype == DT_BF16 ? launch_walk<DT_BF16>(h, a) : launch_walk<DT_FP32>(h, a));
+    const bool bf = h->p.dtype == DT_BF16;
+    cudaError_t le;
+    if (greedy) le = bf ? launch_greedy<DT_BF16>(h, a) : launch_greedy<DT_FP32>(h, a);
+    else if (h->q_probs) le = bf ? launch_walk<DT_BF16, true>(h, a) : launch_walk<DT_FP32, true>(h, a);
+    else le = bf ? launch_walk<DT_BF16, false>(h, a) : launch_walk<DT_FP32, false>(h, a);
+    TP_CUDA(h, le);
     TP_LAUNCHED(h);
     { int rc = profile_mark(h, 1); if (rc) return rc; }
     if (h->profile) h->prof_n[1] += 1;
@@ -435,6 +443,7 @@ int tapout_set_param_i64(tapout_t* h, int key, int64_t v) {
     case TAPOUT_P_TOKEN_UPDATE_ALL: p.token_update_all = v ? 1 : 0; return TAPOUT_OK;
     case TAPOUT_P_DRAFT_GREEDY: p.draft_greedy = v ? 1 : 0; return TAPOUT_OK;
     case TAPOUT_P_VERIFY_GREEDY: p.verify_greedy = v ? 1 : 0; return TAPOUT_OK;
+    case TAPOUT_P_Q_FORMAT: if (v != TAPOUT_Q_LOGITS && v != TAPOUT_Q_PROBS_F32) return TAPOUT_E_INVALID_ARG; h->q_probs = v == TAPOUT_Q_PROBS_F32; return TAPOUT_OK;
     case TAPOUT_P_TOKEN_OUT_STRIDE: if (v < 1) return TAPOUT_E_INVALID_ARG; h->tok_stride = v; return TAPOUT_OK;
     case TAPOUT_P_PROFILE: h->profile = v != 0; return TAPOUT_OK;
     case TAPOUT_P_ROW_SEGMENTS: {
@@ -504,6 +513,7 @@ int tapout_get_param_i64(const tapout_t* h, int key, int64_t* v) {
     case TAPOUT_P_TOKEN_UPDATE_ALL: *v = p.token_update_all; return TAPOUT_OK;
     case TAPOUT_P_DRAFT_GREEDY: *v = p.draft_greedy; return TAPOUT_OK;
     case TAPOUT_P_VERIFY_GREEDY: *v = p.verify_greedy; return TAPOUT_OK;
+    case TAPOUT_P_Q_FORMAT: *v = h->q_probs ? TAPOUT_Q_PROBS_F32 : TAPOUT_Q_LOGITS; return TAPOUT_OK;
     case TAPOUT_P_ROW_SEGMENTS: *v = p.nseg; return TAPOUT_OK;
     case TAPOUT_P_VERIFY_CLUSTER: *v = h->cluster; return TAPOUT_OK;
     case TAPOUT_P_TOKEN_OUT_STRIDE: *v = h->tok_stride; return TAPOUT_OK;
@@ -566,6 +576,7 @@ int tapout_round(tapout_t* h, const void* draft_logits, const void* target_logit
                  uint8_t* out_continue, int32_t* out_accept_len, int32_t* out_next_token) {
     if (!h || !draft_logits || !target_logits || !out_draft_tokens || !out_continue || !out_accept_len || !out_next_token)
         return TAPOUT_E_INVALID_ARG;
+    if (h->q_probs) return TAPOUT_E_UNSUPPORTED;          // one tensor cannot be both the logits drafted from and the probabilities
     if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
     const size_t esz = elem_bytes(h);
     for (int i = 0; i < h->p.K; ++i) {
@@ -583,6 +594,7 @@ int tapout_round_host(tapout_t* h, const void* draft_logits, const void* target_
                       int32_t* out_accept_len, int32_t* out_next_token) {
     if (!h || !draft_logits || !target_logits || !out_draft_tokens || !out_accept_len || !out_next_token)
         return TAPOUT_E_INVALID_ARG;
+    if (h->q_probs) return TAPOUT_E_UNSUPPORTED;
     if (!between_rounds(h)) return TAPOUT_E_BAD_STATE;
     const Params& p = h->p;
     const size_t S = p.S, K = p.K, V = p.V, esz = elem_bytes(h);

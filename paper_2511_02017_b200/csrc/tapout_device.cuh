@@ -607,6 +607,38 @@ __device__ __forceinline__ int pick_residual(const void* prow, const void* qrow,
     }, e0, t, lane);
 }
 
+// PV consecutive draft probabilities (fp32) starting at token e0 (a multiple of 4; the row is 16-byte aligned);
+// tokens at or beyond V have probability 0.
+template <int PV>
+__device__ __forceinline__ void load_qprob_vec(const float* qrow, int V, int e0, float (&q)[PV]) {
+    if (e0 + PV <= V) {
+#pragma unroll
+        for (int k = 0; k < PV / 4; ++k) {
+            const float4 t = __ldg(reinterpret_cast<const float4*>(qrow + e0) + k);
+            q[4 * k] = t.x; q[4 * k + 1] = t.y; q[4 * k + 2] = t.z; q[4 * k + 3] = t.w;
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < PV; ++k) q[k] = (e0 + k < V) ? __ldg(qrow + e0 + k) : 0.f;
+    }
+}
+
+// x ~ norm(max(0, p - q)) inside one chunk with q given as probabilities (read where they are needed: one
+// warp per sequence gets here once).
+template <int DT>
+__device__ __forceinline__ int pick_residual_qprob(const void* prow, const float* qrow, int V, int chunk, float cp, float kp,
+                                                   float beta, double t, int lane) {
+    constexpr int EPL = chunk_elems<DT>() / 32;
+    const int e0 = chunk * chunk_elems<DT>() + lane * EPL;
+    uint4 vp[4];
+    load_lane_block<DT>(prow, V, chunk, lane, vp);
+    return pick_in_block<EPL>([&](int j) {
+        const float wp = ex2_approx(fmaf(lane_block_elem<DT>(vp, j, e0 + j, V), cp, kp));
+        const float q = (e0 + j < V) ? __ldg(qrow + e0 + j) : 0.f;
+        return fmaxf(fmaf(wp, beta, -q), 0.f);
+    }, e0, t, lane);
+}
+
 // In one chunk: how many elements equal the row maximum m, the lowest index of one, and the largest
 // element below m.  Whole warp; every lane returns the same values.
 template <int DT>

@@ -444,11 +444,14 @@ __device__ __forceinline__ int owner_locate(const WalkShared* sh, int which, int
     return cdf_locate<false>(sm_part, nloc, c, mc, SCALED, lane, t, tgt - before, rem);
 }
 
-template <int DT>
-__global__ void __launch_bounds__(kThreads, kWalkResident)
+// QP: the draft distributions are given as normalised fp32 probabilities (q_i(v) is the stored number) instead
+// of logits; the caller's slower format, run at a lower occupancy for the registers its wider loads take.
+template <int DT, bool QP>
+__global__ void __launch_bounds__(kThreads, QP ? 3 : kWalkResident)
 k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
 {
     constexpr int ESZ = Elem<DT>::BYTES;
+    constexpr int QESZ = QP ? 4 : ESZ;
     extern __shared__ float2 sm_part[];                      // partial sums of this CTA's chunks
     __shared__ WalkShared sh;
     cg::cluster_group cl = cg::this_cluster();
@@ -469,7 +472,7 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
     if (cid < n_act) { s = sc.list[(size_t)a.slot * p.S + cid]; n = a.pos; }
     const uint32_t seq = p.seq_offset + (uint32_t)s;
     const char* pbase = reinterpret_cast<const char*>(a.plog) + (size_t)s * a.p_seq * ESZ;
-    const char* qbase = reinterpret_cast<const char*>(a.qlog) + (size_t)s * a.q_seq * ESZ;
+    const char* qbase = reinterpret_cast<const char*>(a.qlog) + (size_t)s * a.q_seq * QESZ;
     const int c0 = (int)(((long long)rank * p.NC) / CS);
     const int c1 = (int)(((long long)(rank + 1) * p.NC) / CS);
     const int nloc = c1 - c0;
@@ -495,9 +498,9 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
             if (ok) {
                 const size_t wo = ((size_t)x_cur * ESZ) & ~(size_t)3;         // the aligned word holding the element
                 cp_async4(&sh.pw[par], prow + wo);
-                cp_async4(&sh.qw[par], qbase + (size_t)i * a.q_pos * ESZ + wo);
+                cp_async4(&sh.qw[par], qbase + (size_t)i * a.q_pos * QESZ + (QP ? (size_t)x_cur * 4 : wo));
             }
-            cp_async8(&sh.dq[par], st.lse_q + (size_t)s * p.K + i);
+            if (!QP) cp_async8(&sh.dq[par], st.lse_q + (size_t)s * p.K + i);
             if (i + 1 < n) x_cur = a.toks[(size_t)s * p.K + i + 1];
         }
         WarpAcc acc;
@@ -519,21 +522,26 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
                 if (lane == 0 && rank == 0) atomicOr(&sc.status[0], 8ull);
                 dec = 0;
             } else {
-                const float zp = word_elem<DT>(sh.pw[par], x), zq = word_elem<DT>(sh.qw[par], x);
+                const float zp = word_elem<DT>(sh.pw[par], x);
                 const double u = (i < kWalkU) ? sh.u[i] : u24_to_double(rng_words(p, seq, a.round, (uint32_t)i, RNG_ACCEPT, 0, 0).x);
                 // p(x) / q(x) = exp((s_p(x) - m_p) - (s_q(x) - lse_q)) / W_p
                 const double dp = ((double)zp - (double)m) * (double)p.inv_Tp;
-                const double logq = (double)zq * (double)p.inv_Tq - sh.dq[par];
-                dec = (u < exp(dp - logq) / W) ? 1 : 0;
+                if (QP) {
+                    // q(x) is the stored number; IEEE division as it stands (q = 0 < p accepts, 0 / 0 rejects)
+                    dec = (u < exp(dp) / W / (double)__uint_as_float(sh.qw[par])) ? 1 : 0;
+                } else {
+                    const double logq = (double)word_elem<DT>(sh.qw[par], x) * (double)p.inv_Tq - sh.dq[par];
+                    dec = (u < exp(dp - logq) / W) ? 1 : 0;
+                }
             }
             if (lane == 0) sh.dec[par] = dec;
             if (dec == 0 && lane == 0) {
                 // rejected: the constants of the residual pass, once, for everybody
-                const double lse_p = (double)m * (double)p.inv_Tp + log(W), lse_q = sh.dq[par];
+                const double lse_p = (double)m * (double)p.inv_Tp + log(W), lse_q = QP ? 0.0 : sh.dq[par];
                 const float kp = (float)(-lse_p * kLog2e), kq = (float)(-lse_q * kLog2e);
                 const double dp = (double)kp + lse_p * kLog2e, dq = (double)kq + lse_q * kLog2e;   // rounding left in kp, kq
                 sh.kp = kp; sh.kq = kq;
-                sh.beta = (float)exp2(dq - dp);      // p = 2^(zc+kp) 2^-dp,  q = 2^(zc+kq) 2^-dq
+                sh.beta = (float)exp2(dq - dp);      // p = 2^(zc+kp) 2^-dp,  q = 2^(zc+kq) 2^-dq (given as it is: dq = 0)
             }
         }
         __syncthreads();                     // the slots of this parity are rewritten two rows on, behind a cluster barrier
@@ -550,13 +558,34 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
     bool from_p = (acc_len == n) && !bad;
     if (!bad && acc_len < n) {
         // residual of the rejected slot: r = max(0, p - q), both rows in one pass (the target row is L2-hot)
-        const char* qrow = qbase + (size_t)acc_len * a.q_pos * ESZ;
+        const char* qrow = qbase + (size_t)acc_len * a.q_pos * QESZ;
         const float kp = sh.kp, kq = sh.kq, beta = sh.beta;  // written with the rejecting decision
         for (int ch = c0 + warp; ch < c1; ch += kWarps) {
             uint4 vp[kVecPerLane], vq[kVecPerLane];
             load_chunk<DT>(prow, p.V, ch, lane, vp);
-            load_chunk<DT>(qrow, p.V, ch, lane, vq);
             float r0 = 0.f, r1 = 0.f;
+            if (QP) {
+                constexpr int PV = Elem<DT>::PV;
+#pragma unroll
+                for (int j = 0; j < kVecPerLane; ++j) {
+                    float q[PV];
+                    load_qprob_vec<PV>(reinterpret_cast<const float*>(qrow), p.V, ch * chunk_elems<DT>() + (j * 32 + lane) * PV, q);
+                    const uint32_t xp[4] = {vp[j].x, vp[j].y, vp[j].z, vp[j].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        if (DT == DT_BF16) {
+                            const float wp0 = ex2_approx(fmaf(__uint_as_float(xp[e] << 16), cp, kp));
+                            const float wp1 = ex2_approx(fmaf(__uint_as_float(xp[e] & 0xffff0000u), cp, kp));
+                            r0 += fmaxf(fmaf(wp0, beta, -q[(2 * e) % PV]), 0.f);
+                            r1 += fmaxf(fmaf(wp1, beta, -q[(2 * e + 1) % PV]), 0.f);
+                        } else {
+                            const float wp0 = ex2_approx(fmaf(__uint_as_float(xp[e]), cp, kp));
+                            r0 += fmaxf(fmaf(wp0, beta, -q[e % PV]), 0.f);
+                        }
+                    }
+                }
+            } else {
+            load_chunk<DT>(qrow, p.V, ch, lane, vq);
 #pragma unroll
             for (int j = 0; j < kVecPerLane; ++j) {
                 const uint32_t xp[4] = {vp[j].x, vp[j].y, vp[j].z, vp[j].w};
@@ -577,6 +606,7 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
                     }
                 }
             }
+            }
             const float tot = warp_sum_f(r0 + r1);
             if (lane == 0) sm_part[ch - c0] = make_float2(0.f, tot);
         }
@@ -591,7 +621,8 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
             double rem;
             const int lc = owner_locate<false>(&sh, 0, rank, CS, sm_part, nloc, 0.f, 0.0, u2, lane, t, rem);
             int tok = -1;
-            if (lc >= 0) tok = pick_residual<DT>(prow, qrow, p.V, c0 + lc, cp, kp, cq, kq, beta, rem, lane);
+            if (lc >= 0) tok = QP ? pick_residual_qprob<DT>(prow, reinterpret_cast<const float*>(qrow), p.V, c0 + lc, cp, kp, beta, rem, lane)
+                                  : pick_residual<DT>(prow, qrow, p.V, c0 + lc, cp, kp, cq, kq, beta, rem, lane);
             if (lane == 0) { sh.i0 = lc; sh.i1 = tok; }
         }
         __syncthreads();

@@ -179,8 +179,15 @@ def run_lockstep(w, rounds, sample=None, device="cuda", logits_fn=None, dev_para
             sum_n += n
 
         # ------------------------------------------------------------ verify
-        dev.verify(draft, target, toks, acc_d, nxt_d)
-        v = ora.verify(Dn, Tn, toks_o)
+        if (dev_params or {}).get("q_format") == tp.Q_PROBS_F32:
+            # the draft distributions handed over as fp32 probabilities: the same bits to both sides
+            qprobs = torch.softmax(draft.float() * float(np.float32(inv_Tq)), dim=2).contiguous()
+            dev.verify(qprobs, target, toks, acc_d, nxt_d)
+            v = ora.verify(qprobs[sample_t].cpu().numpy(), Tn, toks_o)
+            del qprobs
+        else:
+            dev.verify(draft, target, toks, acc_d, nxt_d)
+            v = ora.verify(Dn, Tn, toks_o)
         da = acc_d[sample_t].cpu().numpy()
         dn = nxt_d[sample_t].cpu().numpy()
         patch_acc = []

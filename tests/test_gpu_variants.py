@@ -1,6 +1,9 @@
-"""GPU parity of the greedy variant (draft token = argmax q_i; verification by matching the target's top
-token) against the oracle.  Everything here is integer work: tokens, accepted lengths and final tokens must
-be equal outright, so the lockstep report may show flips for the continue mask only."""
+"""GPU parity of the two variants of the verification step against the oracle.
+
+Greedy (draft token = argmax q_i; verification by matching the target's top token): everything is integer
+work, so tokens, accepted lengths and final tokens must be equal outright and the lockstep report may show
+flips for the continue mask only.  Probability format (tapout_verify given the draft distributions as fp32
+probabilities instead of logits): the usual lockstep bar."""
 import numpy as np
 import pytest
 import torch
@@ -139,3 +142,58 @@ def test_greedy_full_size_round_call_against_separate_calls_and_oracle_sample():
     a.destroy()
     b.destroy()
     torch.cuda.empty_cache()
+
+
+# ------------------------------------------------------------------ draft distributions given as fp32 probabilities
+QPROBS = dict(q_format=1)
+
+
+def _assert_clean(rep):
+    assert rep.ok(), "\n".join(rep.failures[:10]) + "\n" + rep.summary()
+    for k, n in rep.decisions.items():
+        if n >= 200:
+            assert rep.flips[k] <= 0.05 * n, rep.summary()
+    print(rep.summary())
+
+
+@pytest.mark.parametrize("dtype,vocab", [("bf16", 20008), ("fp32", 20004), ("bf16", 1003 + 5), ("fp32", 516)])
+@pytest.mark.parametrize("policy,level", [("ucb1", "seq"), ("ts", "token")])
+def test_probability_format_lockstep(dtype, vocab, policy, level):
+    w = si.Workload("qp", 9, vocab, dtype, 6, 1, 5, policy, level, seed=91, sigma="per_seq:0.2:1.5")
+    rep, dev, _ = run_lockstep(w, 24, device=DEV, logits_fn=peaked_logits, dev_params=QPROBS, orc_params=QPROBS)
+    _assert_clean(rep)
+    assert rep.rows_dev == rep.rows_oracle
+    assert 0.2 < rep.mean_accepted < rep.mean_drafted       # rejections (residual draws) and acceptances both occur
+    dev.destroy()
+
+
+@pytest.mark.parametrize("name,S,rounds", [("throughput", 10, 4), ("batch256_ts", 6, 3), ("shift", 4, 2)])
+def test_probability_format_full_vocab(name, S, rounds):
+    w = si.scaled(si.WORKLOADS[name], n_seq=S)
+    rep, dev, _ = run_lockstep(w, rounds, device=DEV, dev_params=QPROBS, orc_params=QPROBS)
+    _assert_clean(rep)
+    dev.destroy()
+    torch.cuda.empty_cache()
+
+
+def test_probability_format_is_refused_by_the_one_tensor_round_calls_and_checks_alignment():
+    S, V, K = 2, 1032, 2
+    t = tp.Tapout(S, V, K, 1, tp.POLICY_UCB1, tp.LEVEL_SEQ, step_row_stride=K * V, **QPROBS)
+    d = torch.zeros((S, K, V), dtype=torch.bfloat16, device=DEV)
+    p = torch.zeros((S, K + 1, V), dtype=torch.bfloat16, device=DEV)
+    toks = torch.zeros((S, K), dtype=torch.int32, device=DEV)
+    cont = torch.zeros(S, dtype=torch.uint8, device=DEV)
+    acc = torch.zeros(S, dtype=torch.int32, device=DEV)
+    with pytest.raises(tp.TapoutError) as e:
+        t.round(d, p, toks, cont, acc, acc)
+    assert e.value.code == tp.E_UNSUPPORTED
+    tok = torch.zeros(S, dtype=torch.int32, device=DEV)
+    t.draft_step(d[:, 0, :], tok, cont)
+    q = torch.full((S, K, V), 1.0 / V, dtype=torch.float32, device=DEV)
+    with pytest.raises(tp.TapoutError) as e:
+        t.verify(q.view(-1)[1:], p, toks, acc, acc)         # base not 16-byte aligned
+    assert e.value.code == tp.E_ALIGNMENT
+    t.verify(q, p, toks, acc, acc)
+    t.update()
+    assert t.get_param("q_format") == tp.Q_PROBS_F32
+    t.destroy()
