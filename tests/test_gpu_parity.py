@@ -218,6 +218,23 @@ def test_lockstep_full_size_sampled_sequences(name, rounds, n_sample):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("S,V,K,A,policy,level,n_sample", [
+    (3, 1032, 1, 1, "ucb1", "seq", None),        # one draft position: every round stops at once; a single arm
+    (4, 2056, 1, 16, "ts", "token", None),       # the largest arm pool
+    (2, 8, 2, 2, "ucb1", "seq", None),           # a vocabulary of one 16-byte vector
+    (5000, 520, 3, 5, "ucb1", "seq", 8),         # far more sequences than the device has warps for, half a chunk each
+    (2500, 1032, 4, 5, "ts", "token", 6),
+])
+def test_degenerate_and_oversubscribed_shapes(S, V, K, A, policy, level, n_sample):
+    w = si.Workload("edge", S, V, "bf16", K, 1, A, policy, level, seed=73, sigma="per_seq:0.2:1.5")
+    sample = None if n_sample is None else sorted(np.random.default_rng(5).choice(S, size=n_sample, replace=False).tolist())
+    rep, dev, _ = run_lockstep(w, 10, sample=sample, device=DEV, logits_fn=peaked_logits)
+    _assert_clean(rep)
+    st = dev.get_state()
+    assert np.all(st["cnt"].reshape(S, -1, A)[:, 0].sum(axis=1) == 10)      # every sequence was updated every round
+    dev.destroy()
+
+
 @pytest.mark.parametrize("policy", ["ts", "ucb1"])
 def test_token_level_bandits_at_the_papers_draft_cap(policy):
     """gamma = 128, the cap the paper runs with: 128 bandits per sequence at token level, a fixed-length arm in
