@@ -130,7 +130,8 @@ int setup_scratch(tapout* h) {
     int cs = h->cluster_user > 0 ? h->cluster_user : auto_cluster(p.NC, p.S, h->n_sm * kWalkResident);
     if (cs > p.NC) cs = 1;
     for (;; cs >>= 1) {
-        h->walk_smem = sizeof(float2) * (size_t)((p.NC + cs - 1) / cs + 1);
+        h->walk_smem = sizeof(uint4) * kWarps * kStage * kVecPerLane * 32              // staging rings
+                       + sizeof(float2) * (size_t)((p.NC + cs - 1) / cs + 1);         // chunk partials
         if (h->walk_smem > 160 * 1024) return TAPOUT_E_UNSUPPORTED;      // vocabulary too large for the chunk table
         const int fit = (p.dtype == DT_BF16) ? cluster_fits(h, (k_verify_walk<DT_BF16, false>), cs, h->walk_smem)
                                              : cluster_fits(h, (k_verify_walk<DT_FP32, false>), cs, h->walk_smem);

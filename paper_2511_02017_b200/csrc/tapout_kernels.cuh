@@ -54,6 +54,47 @@ __device__ __forceinline__ void stream_chunks(WarpAcc& acc, const void* row, int
     }
 }
 
+// The same share of a row with the loads running ahead of the arithmetic: every lane copies its own four
+// vectors of the next kStage chunks into a ring in shared memory with cp.async and reads back only what it
+// copied itself, so no lane waits for another one and no registers are held for data in flight.  What it
+// buys is bytes in flight per warp: a CTA that has the SM almost to itself (the long drafts at the end of a
+// verification) is otherwise limited to one chunk per warp per memory latency.  ring: this warp's
+// kStage * 128 vectors.  The ragged last chunk of a row takes the plain loads.
+constexpr int kStage = 2;
+template <int DT, bool WANT_T, bool WANT_PART, typename Store>
+__device__ __forceinline__ void stream_chunks_staged(WarpAcc& acc, const void* row, int V, int c0, int c1, int warp, int lane,
+                                                     float c, uint4* ring, Store store) {
+    constexpr int CH = chunk_elems<DT>();
+    constexpr int VPC = CH / Elem<DT>::PV;                // vectors per chunk (128)
+    const int n_whole = V / CH;                           // chunks [0, n_whole) are complete
+    const uint4* rp = reinterpret_cast<const uint4*>(row);
+    auto issue = [&](int ch, int slot) {
+        if (ch < c1 && ch < n_whole) {
+#pragma unroll
+            for (int j = 0; j < kVecPerLane; ++j) cp_async16(ring + (slot * kVecPerLane + j) * 32 + lane, rp + (size_t)ch * VPC + j * 32 + lane);
+        }
+        cp_async_commit();                                // an empty group keeps the count uniform
+    };
+#pragma unroll
+    for (int d = 0; d < kStage; ++d) issue(c0 + warp + d * kWarps, d);
+    int slot = 0;
+    for (int ch = c0 + warp; ch < c1; ch += kWarps) {
+        uint4 v[kVecPerLane];
+        if (ch < n_whole) {
+            cp_async_wait_group<kStage - 1>();
+#pragma unroll
+            for (int j = 0; j < kVecPerLane; ++j) v[j] = ring[(slot * kVecPerLane + j) * 32 + lane];
+        } else {
+            load_chunk<DT>(row, V, ch, lane, v);
+        }
+        const float tot = fold_chunk<DT, WANT_T, WANT_PART>(acc, v, ch, c);
+        if (WANT_PART && lane == 0) store(ch, acc.ref, tot);
+        issue(ch + kStage * kWarps, slot);                // v is in registers: the slot is free
+        slot = (slot + 1 == kStage) ? 0 : slot + 1;
+    }
+    cp_async_wait_all();
+}
+
 // What the finishing warp needs besides Params / State / Scratch.
 // Entry of the list of stopped sequences: the sequence and the number of tokens it drafted, in one word, so
 // that the verification walk learns both from one load.
@@ -452,7 +493,9 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
 {
     constexpr int ESZ = Elem<DT>::BYTES;
     constexpr int QESZ = QP ? 4 : ESZ;
-    extern __shared__ float2 sm_part[];                      // partial sums of this CTA's chunks
+    extern __shared__ uint4 sm_dyn[];                        // per-warp staging rings, then the partial sums of this CTA's chunks
+    uint4* ring = sm_dyn + (threadIdx.x >> 5) * (kStage * kVecPerLane * 32);
+    float2* sm_part = reinterpret_cast<float2*>(sm_dyn + kWarps * kStage * kVecPerLane * 32);
     __shared__ WalkShared sh;
     cg::cluster_group cl = cg::this_cluster();
     const int CS = (int)cl.num_blocks();
@@ -505,10 +548,9 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
         }
         WarpAcc acc;
         acc.init();
-        stream_chunks<DT, false, false>(acc, prow, p.V, c0, c1, warp, lane, cp, [](int, float, float) {});
+        stream_chunks_staged<DT, false, false>(acc, prow, p.V, c0, c1, warp, lane, cp, ring, [](int, float, float) {});
         const float Sw = warp_sum_f(acc.S);
         gather_send(cl, &sh, par, rank, CS, warp, lane, acc.ref, Sw);
-        if (helper) cp_async_wait_all();
         cl.sync();
         if (warp == 0) {
             float m;
@@ -641,8 +683,8 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
         const int par = acc_len & 1;                         // row acc_len - 1 (other parity) may still be read elsewhere
         WarpAcc acc;
         acc.init();
-        stream_chunks<DT, false, true>(acc, prow, p.V, c0, c1, warp, lane, cp,
-                                       [&](int ch, float ref, float tot) { sm_part[ch - c0] = make_float2(ref, tot); });
+        stream_chunks_staged<DT, false, true>(acc, prow, p.V, c0, c1, warp, lane, cp, ring,
+                                              [&](int ch, float ref, float tot) { sm_part[ch - c0] = make_float2(ref, tot); });
         const float Sw = warp_sum_f(acc.S);
         gather_send(cl, &sh, par, rank, CS, warp, lane, acc.ref, Sw);
         cl.sync();                                           // also orders sm_part for warp 0
