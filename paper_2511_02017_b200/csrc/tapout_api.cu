@@ -272,7 +272,8 @@ cudaError_t launch_walk(tapout* h, const WalkArgs& a) {
 
 template <int DT>
 cudaError_t launch_greedy(tapout* h, const WalkArgs& a) {
-    return launch_chained(k_verify_greedy<DT>, (unsigned)h->p.S * (unsigned)h->cluster, kThreads, 0, h->stream,
+    return launch_chained(k_verify_greedy<DT>, (unsigned)h->p.S * (unsigned)h->cluster, kThreads,
+                          sizeof(uint4) * kWarps * kStage * kVecPerLane * 32, h->stream,
                           h->cluster, h->p, h->st, h->sc, a);
 }
 

@@ -61,9 +61,8 @@ __device__ __forceinline__ void stream_chunks(WarpAcc& acc, const void* row, int
 // verification) is otherwise limited to one chunk per warp per memory latency.  ring: this warp's
 // kStage * 128 vectors.  The ragged last chunk of a row takes the plain loads.
 constexpr int kStage = 2;
-template <int DT, bool WANT_T, bool WANT_PART, typename Store>
-__device__ __forceinline__ void stream_chunks_staged(WarpAcc& acc, const void* row, int V, int c0, int c1, int warp, int lane,
-                                                     float c, uint4* ring, Store store) {
+template <int DT, typename Body>
+__device__ __forceinline__ void for_chunks_staged(const void* row, int V, int c0, int c1, int warp, int lane, uint4* ring, Body body) {
     constexpr int CH = chunk_elems<DT>();
     constexpr int VPC = CH / Elem<DT>::PV;                // vectors per chunk (128)
     const int n_whole = V / CH;                           // chunks [0, n_whole) are complete
@@ -87,12 +86,20 @@ __device__ __forceinline__ void stream_chunks_staged(WarpAcc& acc, const void* r
         } else {
             load_chunk<DT>(row, V, ch, lane, v);
         }
-        const float tot = fold_chunk<DT, WANT_T, WANT_PART>(acc, v, ch, c);
-        if (WANT_PART && lane == 0) store(ch, acc.ref, tot);
-        issue(ch + kStage * kWarps, slot);                // v is in registers: the slot is free
+        body(ch, v);
+        issue(ch + kStage * kWarps, slot);                // v has been consumed: the slot is free
         slot = (slot + 1 == kStage) ? 0 : slot + 1;
     }
     cp_async_wait_all();
+}
+
+template <int DT, bool WANT_T, bool WANT_PART, typename Store>
+__device__ __forceinline__ void stream_chunks_staged(WarpAcc& acc, const void* row, int V, int c0, int c1, int warp, int lane,
+                                                     float c, uint4* ring, Store store) {
+    for_chunks_staged<DT>(row, V, c0, c1, warp, lane, ring, [&](int ch, const uint4 (&v)[kVecPerLane]) {
+        const float tot = fold_chunk<DT, WANT_T, WANT_PART>(acc, v, ch, c);
+        if (WANT_PART && lane == 0) store(ch, acc.ref, tot);
+    });
 }
 
 // What the finishing warp needs besides Params / State / Scratch.
@@ -749,6 +756,8 @@ __global__ void __launch_bounds__(kThreads, kWalkResident)
 k_verify_greedy(Params p, State st, Scratch sc, WalkArgs a)
 {
     constexpr int ESZ = Elem<DT>::BYTES;
+    extern __shared__ uint4 sm_dyn[];                        // per-warp staging rings
+    uint4* ring = sm_dyn + (threadIdx.x >> 5) * (kStage * kVecPerLane * 32);
     __shared__ GreedyShared sh;
     cg::cluster_group cl = cg::this_cluster();
     const int CS = (int)cl.num_blocks();
@@ -777,14 +786,12 @@ k_verify_greedy(Params p, State st, Scratch sc, WalkArgs a)
         float ref = neg_inf();
         int best = 0x7fffffff;
         bool nan = false;
-        for (int ch = c0 + warp; ch < c1; ch += kWarps) {
-            uint4 v[kVecPerLane];
-            load_chunk<DT>(prow, p.V, ch, lane, v);
+        for_chunks_staged<DT>(prow, p.V, c0, c1, warp, lane, ring, [&](int ch, const uint4 (&v)[kVecPerLane]) {
             const float lm = lane_max_nan<DT>(v);
             nan = nan || (lm != lm);
             const float M = warp_max_redux(lm);           // NaN lanes are skipped here and reported below
             if (M > ref) { ref = M; best = ch; }
-        }
+        });
         if (__any_sync(0xffffffffu, nan)) ref = __int_as_float(0x7fc00000);
         if (lane < CS) cl.map_shared_rank(&sh, lane)->gather[par][rank][warp] = make_float2(ref, __int_as_float(best));
         cl.sync();
