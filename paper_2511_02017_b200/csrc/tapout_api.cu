@@ -126,24 +126,28 @@ int setup_scratch(tapout* h) {
     if (p.nseg > kMaxSeg) p.nseg = kMaxSeg;
     if (p.nseg > p.NC) p.nseg = p.NC;
 
-    // verify clusters: the requested size, reduced until the device can co-schedule such a cluster
+    // verify clusters: the requested size, reduced until the device can co-schedule such a cluster.  The
+    // kernels are allowed the largest shared memory request this code ever makes before anything asks about
+    // their occupancy with it.
+    constexpr size_t kWalkSmemMax = 160 * 1024;
+    TP_CUDA(h, cudaFuncSetAttribute((k_verify_walk<DT_BF16, false>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWalkSmemMax));
+    TP_CUDA(h, cudaFuncSetAttribute((k_verify_walk<DT_FP32, false>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWalkSmemMax));
+    TP_CUDA(h, cudaFuncSetAttribute((k_verify_walk<DT_BF16, true>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWalkSmemMax));
+    TP_CUDA(h, cudaFuncSetAttribute((k_verify_walk<DT_FP32, true>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWalkSmemMax));
     int cs = h->cluster_user > 0 ? h->cluster_user : auto_cluster(p.NC, p.S, h->n_sm * kWalkResident);
     if (cs > p.NC) cs = 1;
     for (;; cs >>= 1) {
         h->walk_smem = sizeof(uint4) * kWarps * kStage * kVecPerLane * 32              // staging rings
                        + sizeof(float2) * (size_t)((p.NC + cs - 1) / cs + 1);         // chunk partials
-        if (h->walk_smem > 160 * 1024) return TAPOUT_E_UNSUPPORTED;      // vocabulary too large for the chunk table
+        if (h->walk_smem > kWalkSmemMax) {
+            if (cs > 1) continue;                                        // a narrower cluster only makes the table longer
+            return TAPOUT_E_UNSUPPORTED;                                 // vocabulary too large for the chunk table
+        }
         const int fit = (p.dtype == DT_BF16) ? cluster_fits(h, (k_verify_walk<DT_BF16, false>), cs, h->walk_smem)
                                              : cluster_fits(h, (k_verify_walk<DT_FP32, false>), cs, h->walk_smem);
         if (fit > 0 || cs == 1) break;
     }
     h->cluster = cs;
-    if (h->walk_smem > 40 * 1024) {
-        TP_CUDA(h, cudaFuncSetAttribute((k_verify_walk<DT_BF16, false>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
-        TP_CUDA(h, cudaFuncSetAttribute((k_verify_walk<DT_FP32, false>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
-        TP_CUDA(h, cudaFuncSetAttribute((k_verify_walk<DT_BF16, true>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
-        TP_CUDA(h, cudaFuncSetAttribute((k_verify_walk<DT_FP32, true>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->walk_smem));
-    }
 
     if (h->d_scratch) { cudaFree(h->d_scratch); h->d_scratch = nullptr; }
     size_t off = 0;

@@ -258,6 +258,17 @@ def test_vocabulary_beyond_the_register_resident_chunk_table(dtype, vocab):
     torch.cuda.empty_cache()
 
 
+def test_million_token_vocabulary_single_cta_walk():
+    """A row of 1.1 M fp32 logits walked by one CTA per sequence: 2150 chunks, so the walk's table of chunk
+    partials (with its staging rings) needs more shared memory than a kernel gets without asking."""
+    w = si.Workload("huge", 2, 1100008, "fp32", 2, 1, 5, "ucb1", "seq", seed=74)
+    rep, dev, _ = run_lockstep(w, 2, device=DEV, logits_fn=peaked_logits, dev_params=dict(verify_cluster=1))
+    _assert_clean(rep)
+    assert dev.get_param("verify_cluster") == 1
+    dev.destroy()
+    torch.cuda.empty_cache()
+
+
 def test_lockstep_full_size_many_rounds_sampled():
     """The bench workload at full size over enough rounds for UCB1 to leave its exploration phase, with the
     oracle following a handful of sequences."""
