@@ -62,7 +62,7 @@ __device__ __forceinline__ void stream_chunks(WarpAcc& acc, const void* row, int
 // kStage * 128 vectors.  The ragged last chunk of a row takes the plain loads.
 constexpr int kStage = 2;
 template <int DT, typename Body>
-__device__ __forceinline__ void for_chunks_staged(const void* row, int V, int c0, int c1, int warp, int lane, uint4* ring, Body body) {
+__device__ __forceinline__ void for_chunks_staged(const void* row, int V, int first, int c1, int stride, int lane, uint4* ring, Body body) {
     constexpr int CH = chunk_elems<DT>();
     constexpr int VPC = CH / Elem<DT>::PV;                // vectors per chunk (128)
     const int n_whole = V / CH;                           // chunks [0, n_whole) are complete
@@ -75,9 +75,9 @@ __device__ __forceinline__ void for_chunks_staged(const void* row, int V, int c0
         cp_async_commit();                                // an empty group keeps the count uniform
     };
 #pragma unroll
-    for (int d = 0; d < kStage; ++d) issue(c0 + warp + d * kWarps, d);
+    for (int d = 0; d < kStage; ++d) issue(first + d * stride, d);
     int slot = 0;
-    for (int ch = c0 + warp; ch < c1; ch += kWarps) {
+    for (int ch = first; ch < c1; ch += stride) {
         uint4 v[kVecPerLane];
         if (ch < n_whole) {
             cp_async_wait_group<kStage - 1>();
@@ -87,7 +87,7 @@ __device__ __forceinline__ void for_chunks_staged(const void* row, int V, int c0
             load_chunk<DT>(row, V, ch, lane, v);
         }
         body(ch, v);
-        issue(ch + kStage * kWarps, slot);                // v has been consumed: the slot is free
+        issue(ch + kStage * stride, slot);                // v has been consumed: the slot is free
         slot = (slot + 1 == kStage) ? 0 : slot + 1;
     }
     cp_async_wait_all();
@@ -96,7 +96,7 @@ __device__ __forceinline__ void for_chunks_staged(const void* row, int V, int c0
 template <int DT, bool WANT_T, bool WANT_PART, typename Store>
 __device__ __forceinline__ void stream_chunks_staged(WarpAcc& acc, const void* row, int V, int c0, int c1, int warp, int lane,
                                                      float c, uint4* ring, Store store) {
-    for_chunks_staged<DT>(row, V, c0, c1, warp, lane, ring, [&](int ch, const uint4 (&v)[kVecPerLane]) {
+    for_chunks_staged<DT>(row, V, c0 + warp, c1, kWarps, lane, ring, [&](int ch, const uint4 (&v)[kVecPerLane]) {
         const float tot = fold_chunk<DT, WANT_T, WANT_PART>(acc, v, ch, c);
         if (WANT_PART && lane == 0) store(ch, acc.ref, tot);
     });
@@ -335,6 +335,8 @@ __global__ void __launch_bounds__(kThreads, kResident)
 k_draft_stream(Params p, Scratch sc, StepArgs a)
 {
     constexpr int ESZ = Elem<DT>::BYTES;
+    extern __shared__ uint4 sm_ring[];                                          // per-warp staging rings (positions >= 1)
+    uint4* ring = sm_ring + (threadIdx.x >> 5) * (kStage * kVecPerLane * 32);
     const int lane = threadIdx.x & 31;
     const int gw = (int)((blockIdx.x * kThreads + threadIdx.x) >> 5);          // this warp in the grid
     const int n_warps = (int)((gridDim.x * kThreads) >> 5);
@@ -367,11 +369,19 @@ k_draft_stream(Params p, Scratch sc, StepArgs a)
 
         WarpAcc acc;
         acc.init();
-        for (int ch = c0; ch < c1; ++ch) {
-            uint4 v[kVecPerLane];
-            load_chunk<DT>(row, p.V, ch, lane, v);
-            const float tot = fold_chunk<DT, true, true>(acc, v, ch, c);
-            if (lane == 0) part[ch] = make_float2(acc.ref, tot);
+        if (first || FEATURES) {
+            for (int ch = c0; ch < c1; ++ch) {
+                uint4 v[kVecPerLane];
+                load_chunk<DT>(row, p.V, ch, lane, v);
+                const float tot = fold_chunk<DT, true, true>(acc, v, ch, c);
+                if (lane == 0) part[ch] = make_float2(acc.ref, tot);
+            }
+        } else {
+            // later positions: few rows, short items; both chunks of an item are on their way at once
+            for_chunks_staged<DT>(row, p.V, c0, c1, 1, lane, ring, [&](int ch, const uint4 (&v)[kVecPerLane]) {
+                const float tot = fold_chunk<DT, true, true>(acc, v, ch, c);
+                if (lane == 0) part[ch] = make_float2(acc.ref, tot);
+            });
         }
         const float Sw = warp_sum_f(acc.S), Tw = warp_sum_f(acc.T);
         if (lane == 0) {
@@ -786,7 +796,7 @@ k_verify_greedy(Params p, State st, Scratch sc, WalkArgs a)
         float ref = neg_inf();
         int best = 0x7fffffff;
         bool nan = false;
-        for_chunks_staged<DT>(prow, p.V, c0, c1, warp, lane, ring, [&](int ch, const uint4 (&v)[kVecPerLane]) {
+        for_chunks_staged<DT>(prow, p.V, c0 + warp, c1, kWarps, lane, ring, [&](int ch, const uint4 (&v)[kVecPerLane]) {
             const float lm = lane_max_nan<DT>(v);
             nan = nan || (lm != lm);
             const float M = warp_max_redux(lm);           // NaN lanes are skipped here and reported below
