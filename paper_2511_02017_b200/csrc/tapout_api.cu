@@ -256,7 +256,7 @@ int draft_step_impl(tapout* h, const void* logits, int64_t stride, int32_t* out_
     if (h->profile) h->prof_n[0] += 2;
     const unsigned fin_grid = (unsigned)((2 * (long long)h->p.S + 3) / 4);    // two warps per sequence, four per CTA
     const int n_warps = h->grid_rows * kWarps;
-    const size_t ring_bytes = h->pos == 0 ? 0 : sizeof(uint4) * kWarps * kStage * kVecPerLane * 32;   // position 0 loads straight into registers
+    const size_t ring_bytes = sizeof(uint4) * kWarps * kStage * kVecPerLane * 32;   // position 0 loads straight into registers
     TP_CUDA(h, h->p.dtype == DT_BF16
                    ? launch_chained(k_draft_stream<DT_BF16, false>, h->grid_rows, kThreads, ring_bytes, h->stream, 0, h->p, h->sc, a)
                    : launch_chained(k_draft_stream<DT_FP32, false>, h->grid_rows, kThreads, ring_bytes, h->stream, 0, h->p, h->sc, a));

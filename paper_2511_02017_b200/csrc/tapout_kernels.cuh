@@ -369,7 +369,7 @@ k_draft_stream(Params p, Scratch sc, StepArgs a)
 
         WarpAcc acc;
         acc.init();
-        if (first || FEATURES) {
+        if (FEATURES) {
             for (int ch = c0; ch < c1; ++ch) {
                 uint4 v[kVecPerLane];
                 load_chunk<DT>(row, p.V, ch, lane, v);
