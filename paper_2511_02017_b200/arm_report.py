@@ -1,0 +1,98 @@
+"""Single rules, a fixed-length arm and the bandits side by side on synthetic logits.
+
+    python -m paper_2511_02017_b200.arm_report [--workload throughput] [--n-seq 256] [--rounds 200] [--flat]
+
+The paper's comparison (Table 2: Static-6, Max-Confidence, SVIP, AdaEDL against the bandit controllers)
+needs models and datasets; what can be reproduced here is its shape: the same controllers on the same
+seeded draft / target logits, reporting per controller the mean drafted length |X|, the mean accepted
+length m = |Y|, the acceptance rate |Y| / |X|, and the logit rows read per emitted token (the cost this
+library can see; wall-clock speed-up needs the model forwards).  Runs on the device through the C ABI.
+By default the rows are the peaked variant of the workload (top-1 probabilities spread over (0, 1), so the
+rules differ); --flat takes the workload's own rows, on which four of the five rules stop at once.
+"""
+import argparse
+import json
+
+import numpy as np
+import torch
+
+from . import binding as tp
+from . import synth_inputs as si
+
+RULES = [("Max-Confidence", tp.RULE_MAXCONF), ("SVIP", tp.RULE_SVIP), ("AdaEDL", tp.RULE_ADAEDL),
+         ("SVIP-Difference", tp.RULE_SVIPDIFF), ("LogitMargin", tp.RULE_MARGIN)]
+
+
+def run(w, rounds, gen, device, n_arms, policy, level, arms=None, static_len=None):
+    """One controller over `rounds` rounds; returns its summary."""
+    k_max = static_len if static_len else w.k_max
+    ww = si.scaled(w, n_arms=n_arms, policy=policy, level=level)
+    params = dict(token_out_stride=w.k_max)
+    if arms is not None:
+        params["arms"] = arms
+    dev = tp.Tapout.from_workload(ww, **params)
+    S, K = w.n_seq, w.k_max
+    toks = torch.full((S, K), -1, dtype=torch.int32, device=device)
+    tok = torch.empty(S, dtype=torch.int32, device=device)
+    cont = torch.empty(S, dtype=torch.uint8, device=device)
+    acc = torch.empty(S, dtype=torch.int32, device=device)
+    nxt = torch.empty(S, dtype=torch.int32, device=device)
+    sum_n = sum_a = 0
+    for rnd in range(rounds):
+        d, t = gen(w, rnd, device)
+        if static_len:
+            # a fixed-length arm drafts exactly static_len tokens: the caller simply stops asking after that
+            toks.fill_(-1)
+            for i in range(static_len):
+                dev.draft_step(d[:, i, :], tok, cont)
+                toks[:, i] = tok
+            dev.verify(d, t, toks, acc, nxt)
+            dev.update()
+        else:
+            dev.round(d, t, toks, cont, acc, nxt)
+        st = dev.get_state()
+        sum_n += int(st["n_drafted"].sum())
+        sum_a += int(acc.sum().item())
+    rows = dev.get_status()
+    plays = dev.get_state()["cnt"].reshape(S, -1, n_arms).sum(axis=(0, 1))
+    dev.destroy()
+    n_rounds = rounds * S
+    total_rows = rows["rows_draft"] + rows["rows_target"] + rows["rows_residual"]
+    return dict(mean_drafted=sum_n / n_rounds, mean_accepted=sum_a / n_rounds, accept_rate=sum_a / max(1, sum_n),
+                rows_per_token=total_rows / (sum_a + n_rounds), plays=plays.tolist(), k=k_max)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="throughput", choices=sorted(si.WORKLOADS))
+    ap.add_argument("--n-seq", type=int, default=256)
+    ap.add_argument("--rounds", type=int, default=200)
+    ap.add_argument("--flat", action="store_true")
+    ap.add_argument("--static-k", type=int, default=6)
+    ap.add_argument("--json", action="store_true")
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("arm_report runs on the device: no CUDA device visible")
+    w = si.scaled(si.WORKLOADS[args.workload], n_seq=args.n_seq)
+    gen = si.round_logits if args.flat else si.peaked_round_logits
+    device = "cuda"
+    out = {}
+    out["Static-%d" % min(args.static_k, w.k_max)] = run(w, args.rounds, gen, device, 1, "ucb1", "seq", arms=[tp.RULE_STATIC],
+                                                          static_len=min(args.static_k, w.k_max))
+    for name, rule in RULES:
+        out[name] = run(w, args.rounds, gen, device, 1, "ucb1", "seq", arms=[rule])
+    for name, policy, level in (("Seq-UCB1", "ucb1", "seq"), ("Seq-UCB-Tuned", "ucb_tuned", "seq"), ("Seq-TS", "ts", "seq"),
+                                ("Token-UCB1", "ucb1", "token"), ("Token-TS", "ts", "token")):
+        out[name] = run(w, args.rounds, gen, device, 5, policy, level)
+    if args.json:
+        print(json.dumps(out))
+        return
+    print("%s, %d sequences, %d rounds, %s rows, k_max %d" % (w.name, w.n_seq, args.rounds, "flat" if args.flat else "peaked", w.k_max))
+    print("%-16s %9s %9s %9s %12s  %s" % ("controller", "|X|", "m = |Y|", "|Y|/|X|", "rows/token", "plays per arm"))
+    for name, r in out.items():
+        print("%-16s %9.3f %9.3f %9.3f %12.3f  %s" % (name, r["mean_drafted"], r["mean_accepted"], r["accept_rate"],
+                                                       r["rows_per_token"], r["plays"] if len(r["plays"]) > 1 else ""))
+
+
+if __name__ == "__main__":
+    main()

@@ -145,6 +145,23 @@ def round_logits(w: Workload, rnd: int, device="cpu"):
     return draft, target
 
 
+def peaked_round_logits(w: Workload, rnd: int, device="cpu"):
+    """round_logits with one token per row lifted by U[6, 16] (the draft's by 0.9 of that): the rows of the
+    configs are flat (top-1 probability about 1e-3), these have top-1 probabilities spread over (0, 1), so that
+    every stop rule fires on some rows and drafts of every length occur.  Same shapes, dtype and seeding."""
+    d, t = round_logits(w, rnd, device)
+    g = torch.Generator(device="cpu")
+    g.manual_seed(1234 + rnd)
+    S, K, V = w.n_seq, w.k_max, w.vocab
+    idx = torch.randint(0, V, (S, K + 1), generator=g).to(device)
+    lift = (6 + 10 * torch.rand((S, K + 1), generator=g)).to(device)
+    tt = t.float()
+    tt.scatter_add_(2, idx.unsqueeze(-1), lift.unsqueeze(-1))
+    dd = d.float()
+    dd.scatter_add_(2, idx[:, :K].unsqueeze(-1), (lift[:, :K] * 0.9).unsqueeze(-1))
+    return dd.to(d.dtype), tt.to(t.dtype)
+
+
 def to_numpy_bits(t: torch.Tensor) -> np.ndarray:
     """Host copy as the arrays the oracle reads: float32, or uint16 holding bf16 bits."""
     t = t.detach().cpu().contiguous()

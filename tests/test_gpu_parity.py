@@ -25,19 +25,9 @@ def _assert_clean(rep, max_flip_rate=0.05):
 
 
 def peaked_logits(w, rnd, device):
-    """The workload's rows with one token per row lifted by U[6,16]: top-1 probabilities then spread over
-    (0,1) so that every stop rule fires on some rows and drafts of every length occur."""
-    d, t = si.round_logits(w, rnd, device)
-    g = torch.Generator(device="cpu")
-    g.manual_seed(1234 + rnd)
-    S, K, V = w.n_seq, w.k_max, w.vocab
-    idx = torch.randint(0, V, (S, K + 1), generator=g).to(device)
-    lift = (6 + 10 * torch.rand((S, K + 1), generator=g)).to(device)
-    tt = t.float()
-    tt.scatter_add_(2, idx.unsqueeze(-1), lift.unsqueeze(-1))
-    dd = d.float()
-    dd.scatter_add_(2, idx[:, :K].unsqueeze(-1), (lift[:, :K] * 0.9).unsqueeze(-1))
-    return dd.to(d.dtype), tt.to(t.dtype)
+    """The workload's rows with one token per row lifted, so that every stop rule fires on some rows and
+    drafts of every length occur (the recipe lives with the other input generators)."""
+    return si.peaked_round_logits(w, rnd, device)
 
 
 # ------------------------------------------------------------------ row statistics kernel

@@ -197,3 +197,17 @@ def test_probability_format_is_refused_by_the_one_tensor_round_calls_and_checks_
     t.update()
     assert t.get_param("q_format") == tp.Q_PROBS_F32
     t.destroy()
+
+
+# ------------------------------------------------------------------ controllers side by side
+def test_arm_report_runs_every_controller():
+    """The report module: a fixed-length arm drafts exactly its length, a single-rule pool plays one arm, the
+    bandits spread their plays; rows per emitted token are what the status counters say."""
+    from paper_2511_02017_b200 import arm_report
+    w = si.Workload("rep", 12, 4104, "bf16", 6, 1, 5, "ucb1", "seq", seed=95)
+    r = arm_report.run(w, 6, si.peaked_round_logits, DEV, 1, "ucb1", "seq", arms=[tp.RULE_STATIC], static_len=4)
+    assert r["mean_drafted"] == 4.0 and 0 <= r["mean_accepted"] <= 4.0 and r["plays"] == [12 * 6]
+    r = arm_report.run(w, 6, si.peaked_round_logits, DEV, 1, "ucb1", "seq", arms=[tp.RULE_MARGIN])
+    assert 1.0 <= r["mean_drafted"] <= 6.0 and r["plays"] == [12 * 6]
+    r = arm_report.run(w, 10, si.peaked_round_logits, DEV, 5, "ts", "token")
+    assert len(r["plays"]) == 5 and sum(r["plays"]) >= 12 * 10 and 1.0 <= r["rows_per_token"] <= 3.0
