@@ -1,14 +1,16 @@
-// Kernels of libtapout (sm_100a).  The two streaming kernels read each needed logit row from HBM
-// exactly once with 128-bit coalesced loads; everything per-row that is scalar runs in double.
+// Kernels of libtapout (sm_100a).  The streaming kernels read each needed logit row from HBM exactly once,
+// 16 bytes per lane and 512 contiguous bytes per warp instruction, staged two chunks ahead through per-warp
+// cp.async rings in shared memory; everything per-row that is scalar runs in double.
 //
 //   k_draft_stream  first kernel of a draft position: a persistent grid of independent warps, each
 //                   reducing one segment of one drafted row (ticket-scheduled), leaving a segment
 //                   record and per-chunk partial sums.
-//   k_draft_finish  second kernel: one warp per sequence combines the segments of its row (features,
-//                   token draw, stop rule, bookkeeping, lists for the next position).
+//   k_draft_finish  second kernel: two warps per sequence combine the segments of its row (one: features,
+//                   stop rule, bookkeeping, lists for the next position; the other: the token draw).
 //   k_verify_walk   one thread-block cluster per sequence: every CTA streams its slice of the target
 //                   row, the per-warp partial sums are exchanged through distributed shared memory,
 //                   and all CTAs take the same accept / reject decision before the next row.
+//   k_verify_greedy the same walk for verification by matching the target's top token (maximum only).
 //   k_update        rewards, arm statistics, AdaEDL, and the arm choices of the next round.
 #pragma once
 
@@ -21,7 +23,7 @@ namespace tpo {
 namespace cg = cooperative_groups;
 
 constexpr int kMaxCluster = 8;           // portable cluster size limit
-constexpr int kFinishThreads = 128;       // k_draft_finish: four rows per CTA, no register ceiling
+constexpr int kFinishThreads = 128;       // k_draft_finish: two sequences (two warps each) per CTA, no register ceiling
 constexpr int kResident = 4;              // k_draft_stream CTAs resident per SM (64 registers per thread)
 constexpr int kWalkResident = 5;          // k_verify_walk CTAs resident per SM (48 registers: its fold keeps no entropy sums)
 
@@ -39,22 +41,8 @@ __device__ __forceinline__ int segments_for(const Params& p, int n_rows, int n_w
     return max(1, min(nseg, cap));
 }
 
-// One warp's share of the chunks [c0, c1) of a row: chunk c0 + warp, then every kWarps-th.  Loads are not
-// staged ahead: with four CTAs resident per SM the other warps cover the latency, and the registers a
-// second buffer would take cost more than it gains.  store(ch, ref, total) receives the per-chunk partial
-// sum when WANT_PART.
-template <int DT, bool WANT_T, bool WANT_PART, typename Store>
-__device__ __forceinline__ void stream_chunks(WarpAcc& acc, const void* row, int V, int c0, int c1, int warp, int lane,
-                                              float c, Store store) {
-    for (int ch = c0 + warp; ch < c1; ch += kWarps) {
-        uint4 v[kVecPerLane];
-        load_chunk<DT>(row, V, ch, lane, v);
-        const float tot = fold_chunk<DT, WANT_T, WANT_PART>(acc, v, ch, c);
-        if (WANT_PART && lane == 0) store(ch, acc.ref, tot);
-    }
-}
-
-// The same share of a row with the loads running ahead of the arithmetic: every lane copies its own four
+// A warp's share of the chunks of a row (chunk `first`, then every stride-th, below c1) with the loads
+// running ahead of the arithmetic: every lane copies its own four
 // vectors of the next kStage chunks into a ring in shared memory with cp.async and reads back only what it
 // copied itself, so no lane waits for another one and no registers are held for data in flight.  What it
 // buys is bytes in flight per warp: a CTA that has the SM almost to itself (the long drafts at the end of a
@@ -324,11 +312,12 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
 }
 
 // ============================================================================================
-// One draft position (Algorithm 1, loop body) for every sequence still drafting.  Work item =
-// (row, segment of the row); the persistent grid strides over the items.  Per item the CTA leaves a
-// SegRec and, per 2 KB chunk, the chunk's partial softmax sum (for the inverse-CDF draw); a per-row
-// counter tells the CTA that reduced the last segment to finish the row.  No CTA ever waits for
-// another one.  FEATURES: rows 0 .. n_fixed-1 instead of the drafting list, features to out_feat.
+// One draft position (Algorithm 1, loop body) for every sequence still drafting, first half: the
+// streaming.  Work item = (row, segment of the row), one warp each; the persistent grid takes the first
+// items by position and the rest by ticket.  Per item a warp leaves a SegRec and, per 2 KB chunk, the
+// chunk's partial softmax sum (for the inverse-CDF draw); k_draft_finish, the next kernel in the stream,
+// combines them.  No warp ever waits for another one.  FEATURES: rows 0 .. n_fixed-1 instead of the
+// drafting list.
 // ============================================================================================
 template <int DT, bool FEATURES>
 __global__ void __launch_bounds__(kThreads, kResident)
@@ -443,7 +432,6 @@ constexpr int kWalkU = 32;
 struct WalkShared {
     float2 gather[2][kMaxCluster][kWarps];   // per-warp (reference, sum) of every CTA of the cluster, by row parity
     double ctot[2][kMaxCluster];             // per-CTA totals of the final draw: [0] residual, [1] target row
-    float2 wrec[kWarps];
     double dq[2];                            // the draft row's lse, by row parity
     double u[kWalkU];                        // uniforms of the accept tests of the first rows
     uint32_t pw[2], qw[2];                   // the words holding z_p(x), z_q(x) of the row's draft token
