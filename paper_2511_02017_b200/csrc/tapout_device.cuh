@@ -665,55 +665,67 @@ __device__ __forceinline__ void scan_top_block(const uint4 (&v)[4], int V, int c
     below = warp_max_f(b);
 }
 
-// ------------------------------------------------------------------ bandits (double, one thread)
-__device__ __forceinline__ int argmax_first(const double* val, int A) {
+// ------------------------------------------------------------------ bandits (double; lane a holds arm a)
+// The statistics of a bandit sit one arm per lane (N, R, R2 of arm `lane`; lanes >= A hold nothing), so
+// that they are fetched in one trip and every arm's value is worked out at once; the arithmetic per arm
+// is the scalar formula as printed.  Every lane returns the chosen arm.
+
+// First index of the largest value, scanned in arm order with a strict comparison (ties to the lowest index).
+__device__ __forceinline__ int argmax_first_lanes(double val, int A) {
     int best = 0;
-    for (int a = 1; a < A; ++a) if (val[a] > val[best]) best = a;
+    double vbest = __shfl_sync(0xffffffffu, val, 0);
+    for (int a = 1; a < A; ++a) {
+        const double va = __shfl_sync(0xffffffffu, val, a);
+        if (va > vbest) { best = a; vbest = va; }
+    }
     return best;
 }
 
+__device__ __forceinline__ unsigned long long plays_plus_one(uint32_t N, int A, int lane) {
+    unsigned long long t = lane < A ? N : 0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    return t + 1;
+}
+
 // UCB1 (Section 3.3): mu_a + sqrt(c2 ln t / N_a), t = 1 + sum N; unplayed arms first.
-__device__ inline int ucb1_select(const uint32_t* N, const double* R, int A, double c2) {
-    for (int a = 0; a < A; ++a) if (N[a] == 0) return a;
-    unsigned long long t = 1;
-    for (int a = 0; a < A; ++a) t += N[a];
-    const double lt = log((double)t);
-    double val[kMaxArms];
-    for (int a = 0; a < A; ++a) val[a] = R[a] / (double)N[a] + sqrt(c2 * lt / (double)N[a]);
-    return argmax_first(val, A);
+__device__ inline int ucb1_select(uint32_t N, double R, int A, double c2, int lane) {
+    const unsigned unplayed = __ballot_sync(0xffffffffu, lane < A && N == 0);
+    if (unplayed) return __ffs(unplayed) - 1;
+    const double lt = log((double)plays_plus_one(N, A, lane));
+    const double val = lane < A ? R / (double)N + sqrt(c2 * lt / (double)N) : 0.0;
+    return argmax_first_lanes(val, A);
 }
 
 // UCB-Tuned (Section 3.3): mu_a + sqrt((ln t / N_a) min(1/4, V_a)), V_a = var_a + sqrt(2 ln t / N_a).
-__device__ inline int ucb_tuned_select(const uint32_t* N, const double* R, const double* R2, int A) {
-    for (int a = 0; a < A; ++a) if (N[a] == 0) return a;
-    unsigned long long t = 1;
-    for (int a = 0; a < A; ++a) t += N[a];
-    const double lt = log((double)t);
-    double val[kMaxArms];
-    for (int a = 0; a < A; ++a) {
-        const double n = (double)N[a];
-        const double mu = R[a] / n;
-        const double var = R2[a] / n - mu * mu;
+__device__ inline int ucb_tuned_select(uint32_t N, double R, double R2, int A, int lane) {
+    const unsigned unplayed = __ballot_sync(0xffffffffu, lane < A && N == 0);
+    if (unplayed) return __ffs(unplayed) - 1;
+    const double lt = log((double)plays_plus_one(N, A, lane));
+    double val = 0.0;
+    if (lane < A) {
+        const double n = (double)N;
+        const double mu = R / n;
+        const double var = R2 / n - mu * mu;
         const double Va = var + sqrt(2.0 * lt / n);
         const double cap = Va < 0.25 ? Va : 0.25;
-        val[a] = mu + sqrt((lt / n) * cap);
+        val = mu + sqrt((lt / n) * cap);
     }
-    return argmax_first(val, A);
+    return argmax_first_lanes(val, A);
 }
 
 // Gaussian Thompson Sampling (sequence level): conjugate normal posterior, Box-Muller draw.
-__device__ inline int ts_gauss_select(const Params& p, const uint32_t* N, const double* R, uint32_t seq,
-                                      uint32_t round, uint32_t pos) {
-    double val[kMaxArms];
-    for (int a = 0; a < p.A; ++a) {
-        const double var_n = 1.0 / (1.0 / p.ts_var0 + (double)N[a] / p.ts_noise_var);
-        const double mu_n = var_n * (p.ts_mu0 / p.ts_var0 + R[a] / p.ts_noise_var);
-        const uint4 w = rng_words(p, seq, round, pos, RNG_BANDIT, (uint32_t)a, 0);
+__device__ inline int ts_gauss_select(const Params& p, uint32_t N, double R, uint32_t seq, uint32_t round, uint32_t pos, int lane) {
+    double val = 0.0;
+    if (lane < p.A) {
+        const double var_n = 1.0 / (1.0 / p.ts_var0 + (double)N / p.ts_noise_var);
+        const double mu_n = var_n * (p.ts_mu0 / p.ts_var0 + R / p.ts_noise_var);
+        const uint4 w = rng_words(p, seq, round, pos, RNG_BANDIT, (uint32_t)lane, 0);
         const double u1 = u24_to_double(w.x), u2 = u24_to_double(w.y);
         const double z = sqrt(-2.0 * log(1.0 - u1)) * cos(6.283185307179586476925 * u2);
-        val[a] = mu_n + sqrt(var_n) * z;
+        val = mu_n + sqrt(var_n) * z;
     }
-    return argmax_first(val, p.A);
+    return argmax_first_lanes(val, p.A);
 }
 
 // Beta(alpha, beta), integer parameters, as the alpha-th smallest of n = alpha+beta-1 uniforms
@@ -780,13 +792,13 @@ __device__ inline uint32_t beta_order_stat_warp(const Params& p, uint32_t alpha,
 }
 
 // Beta-Bernoulli Thompson Sampling (token level).  Whole warp; every lane returns the arm.
-__device__ inline int ts_beta_select_warp(const Params& p, const uint32_t* N, const double* R, uint32_t seq,
+__device__ inline int ts_beta_select_warp(const Params& p, uint32_t N, double R, uint32_t seq,
                                           uint32_t round, uint32_t pos, uint32_t* hist, int lane) {
     int best = 0;
     uint32_t best_v = 0;
     for (int a = 0; a < p.A; ++a) {
-        const uint32_t succ = (uint32_t)R[a];
-        const uint32_t fail = N[a] - succ;
+        const uint32_t succ = (uint32_t)__shfl_sync(0xffffffffu, R, a);
+        const uint32_t fail = __shfl_sync(0xffffffffu, N, a) - succ;
         const uint32_t v = beta_order_stat_warp(p, p.ts_a0 + succ, p.ts_b0 + fail, seq, round, pos, (uint32_t)a, hist, lane);
         if (a == 0 || v > best_v) { best = a; best_v = v; }
     }

@@ -432,6 +432,8 @@ constexpr int kWalkU = 32;
 struct WalkShared {
     float2 gather[2][kMaxCluster][kWarps];   // per-warp (reference, sum) of every CTA of the cluster, by row parity
     double ctot[2][kMaxCluster];             // per-CTA totals of the final draw: [0] residual, [1] target row
+    char pad_[64];                           // keeps what follows 64 bytes into a 128-byte segment: measured, the walk is 4 % slower with the
+                                             // accept-test fields starting on a 128-byte boundary (with no padding as with 128 bytes of it)
     double dq[2];                            // the draft row's lse, by row parity
     double u[kWalkU];                        // uniforms of the accept tests of the first rows
     uint32_t pw[2], qw[2];                   // the words holding z_p(x), z_q(x) of the row's draft token
@@ -830,29 +832,23 @@ k_verify_greedy(Params p, State st, Scratch sc, WalkArgs a)
 }
 
 // ============================================================================================
-// Bandit arm for one slot (sequence level: slot 0; token level: slot = draft position), Section 3.3.
-// Whole warp; every lane returns the arm.
+// Bandit arm for one slot (sequence level: slot 0; token level: slot = draft position), Section 3.3, from
+// the statistics held one arm per lane.  Whole warp; every lane returns the arm.
 // ============================================================================================
-__device__ __forceinline__ int select_arm(const Params& p, const State& st, int s, int slot, uint32_t round,
+__device__ __forceinline__ int select_arm(const Params& p, uint32_t N, double R, double R2, int s, int slot, uint32_t round,
                                           uint32_t* hist, int lane) {
-    const size_t o = ((size_t)s * p.P + slot) * p.A;
     const uint32_t seq = p.seq_offset + (uint32_t)s;
-    if (p.policy == 1 && p.level == 1)
-        return ts_beta_select_warp(p, st.cnt + o, st.rsum + o, seq, round, (uint32_t)slot, hist, lane);
-    int arm = 0;
-    if (lane == 0) {
-        if (p.policy == 0) arm = ucb1_select(st.cnt + o, st.rsum + o, p.A, p.ucb_c2);
-        else if (p.policy == 2) arm = ucb_tuned_select(st.cnt + o, st.rsum + o, st.rsum2 + o, p.A);
-        else arm = ts_gauss_select(p, st.cnt + o, st.rsum + o, seq, round, 0u);
-    }
-    return __shfl_sync(0xffffffffu, arm, 0);
+    if (p.policy == 1 && p.level == 1) return ts_beta_select_warp(p, N, R, seq, round, (uint32_t)slot, hist, lane);
+    if (p.policy == 0) return ucb1_select(N, R, p.A, p.ucb_c2, lane);
+    if (p.policy == 2) return ucb_tuned_select(N, R, R2, p.A, lane);
+    return ts_gauss_select(p, N, R, seq, round, 0u, lane);
 }
 
 // Arm of round `round` for one bandit (sequence s, slot k; sequence level has the single slot 0, whose arm
 // serves every position), and, from the warp of slot 0, the round's bookkeeping.
-__device__ __forceinline__ void begin_round(const Params& p, const State& st, const Scratch& sc, int s, int k,
-                                            uint32_t round, uint32_t* hist, int lane, bool reset_counts) {
-    const int arm = select_arm(p, st, s, k, round, hist, lane);
+__device__ __forceinline__ void begin_round(const Params& p, const State& st, const Scratch& sc, uint32_t N, double R, double R2,
+                                            int s, int k, uint32_t round, uint32_t* hist, int lane, bool reset_counts) {
+    const int arm = select_arm(p, N, R, R2, s, k, round, hist, lane);
     if (p.level == 0) { for (int kk = lane; kk < p.K; kk += 32) st.arm[(size_t)s * p.K + kk] = arm; }
     else if (lane == 0) st.arm[(size_t)s * p.K + k] = arm;
     if (k == 0 && lane == 0) {
@@ -864,8 +860,10 @@ __device__ __forceinline__ void begin_round(const Params& p, const State& st, co
 
 // update(pi, |Y|, |X|, gamma): rewards, arm statistics, AdaEDL; then the arms of the next round.  One warp
 // per bandit (sequence, slot): the Beta draws of token-level Thompson Sampling cost O(plays) each, so the
-// slots of a sequence must not queue behind one another.  The drafted and accepted lengths are read by all
-// warps of a sequence and therefore left alone here: position 0 of the next round rewrites them.
+// slots of a sequence must not queue behind one another.  Lane a holds the statistics of arm a: one trip to
+// memory fetches them together with the round's outcome, the lane of the played arm applies the reward, and
+// the next arm is chosen from the registers.  The drafted and accepted lengths are read by all warps of a
+// sequence and therefore left alone here: position 0 of the next round rewrites them.
 __global__ void __launch_bounds__(128)
 k_update(Params p, State st, Scratch sc, uint32_t next_round)
 {
@@ -876,39 +874,43 @@ k_update(Params p, State st, Scratch sc, uint32_t next_round)
     pdl_trigger();
     pdl_wait();
     if (s >= p.S) return;
-    if (lane == 0) {
-        const int n = st.n_drafted[s], a = st.accept_len[s];
-        if (n > 0) {
-            if (p.level == 0) {
-                const double r = p.reward_kind ? ((double)a / (double)p.K)
-                                               : (p.reward_alpha * ((double)a / (double)p.K) +
-                                                  (1.0 - p.reward_alpha) * ((double)a / (double)n));
-                const size_t o = (size_t)s * p.A + st.arm[(size_t)s * p.K];
-                st.cnt[o] += 1; st.rsum[o] += r; st.rsum2[o] += r * r;
-                st.reward[s] = r;
-            } else {
-                const int last = p.token_update_all ? n : min(a + 1, n);
-                if (k < last) {
-                    const double r = (k < a) ? 1.0 : 0.0;
-                    const size_t o = ((size_t)s * p.K + k) * p.A + st.arm[(size_t)s * p.K + k];
-                    st.cnt[o] += 1; st.rsum[o] += r; st.rsum2[o] += r * r;
-                }
-                if (k == 0) st.reward[s] = (double)a;
-            }
-            if (k == 0) {
-                // AdaEDL, as printed: lambda <- b2*lambda + (1-b2)*(lambda + eps*sign(alpha - r))
-                const double r = (double)a / (double)n;
-                const double d = p.ada_alpha - r;
-                const double sgn = (double)((d > 0.0) - (d < 0.0));
-                st.acc_rate[s] = p.ada_beta1 * st.acc_rate[s] + (1.0 - p.ada_beta1) * r;
-                st.lambda[s] = p.ada_beta2 * st.lambda[s] + (1.0 - p.ada_beta2) * (st.lambda[s] + p.ada_eps * sgn);
-            }
-        } else if (k == 0) {
-            st.reward[s] = 0.0;
+    const size_t o = ((size_t)s * p.P + k) * p.A;
+    uint32_t N = 0;
+    double R = 0.0, R2 = 0.0;
+    if (lane < p.A) { N = st.cnt[o + lane]; R = st.rsum[o + lane]; R2 = st.rsum2[o + lane]; }
+    const int n = st.n_drafted[s], a = st.accept_len[s];
+    const int played = st.arm[(size_t)s * p.K + k];        // sequence level: k = 0, the arm of every position
+    double lambda = 0.0, acc_rate = 0.0;
+    if (k == 0 && lane == 0) { lambda = st.lambda[s]; acc_rate = st.acc_rate[s]; }
+    if (n > 0) {
+        double r = 0.0;
+        bool rewarded;
+        if (p.level == 0) {
+            r = p.reward_kind ? ((double)a / (double)p.K)
+                              : (p.reward_alpha * ((double)a / (double)p.K) + (1.0 - p.reward_alpha) * ((double)a / (double)n));
+            rewarded = true;
+        } else {
+            const int last = p.token_update_all ? n : min(a + 1, n);
+            rewarded = k < last;
+            r = (k < a) ? 1.0 : 0.0;
         }
+        if (rewarded && lane == played) {
+            N += 1; R += r; R2 += r * r;
+            st.cnt[o + lane] = N; st.rsum[o + lane] = R; st.rsum2[o + lane] = R2;
+        }
+        if (k == 0 && lane == 0) {
+            st.reward[s] = p.level == 0 ? r : (double)a;
+            // AdaEDL, as printed: lambda <- b2*lambda + (1-b2)*(lambda + eps*sign(alpha - r))
+            const double ra = (double)a / (double)n;
+            const double d = p.ada_alpha - ra;
+            const double sgn = (double)((d > 0.0) - (d < 0.0));
+            st.acc_rate[s] = p.ada_beta1 * acc_rate + (1.0 - p.ada_beta1) * ra;
+            st.lambda[s] = p.ada_beta2 * lambda + (1.0 - p.ada_beta2) * (lambda + p.ada_eps * sgn);
+        }
+    } else if (k == 0 && lane == 0) {
+        st.reward[s] = 0.0;
     }
-    __syncwarp();
-    begin_round(p, st, sc, s, k, next_round, hist[warp], lane, false);
+    begin_round(p, st, sc, N, R, R2, s, k, next_round, hist[warp], lane, false);
 }
 
 // Start of a round without an update before it (a new handle, a changed parameter, restored state):
@@ -924,8 +926,11 @@ k_begin_round(Params p, State st, Scratch sc, uint32_t round, int reset_adaedl)
     pdl_wait();
     if (s >= p.S) return;
     if (reset_adaedl && k == 0 && lane == 0) { st.lambda[s] = p.ada_lambda0; st.acc_rate[s] = p.ada_acc0; }
-    __syncwarp();
-    begin_round(p, st, sc, s, k, round, hist[warp], lane, true);
+    const size_t o = ((size_t)s * p.P + k) * p.A;
+    uint32_t N = 0;
+    double R = 0.0, R2 = 0.0;
+    if (lane < p.A) { N = st.cnt[o + lane]; R = st.rsum[o + lane]; R2 = st.rsum2[o + lane]; }
+    begin_round(p, st, sc, N, R, R2, s, k, round, hist[warp], lane, true);
 }
 
 // After tapout_set_state in the middle of a round: the drafting list of position `pos` and the list of
