@@ -324,7 +324,7 @@ __global__ void __launch_bounds__(kThreads, kResident)
 k_draft_stream(Params p, Scratch sc, StepArgs a)
 {
     constexpr int ESZ = Elem<DT>::BYTES;
-    extern __shared__ uint4 sm_ring[];                                          // per-warp staging rings (positions >= 1)
+    extern __shared__ __align__(128) uint4 sm_ring[];             // per-warp staging rings
     uint4* ring = sm_ring + (threadIdx.x >> 5) * (kStage * kVecPerLane * 32);
     const int lane = threadIdx.x & 31;
     const int gw = (int)((blockIdx.x * kThreads + threadIdx.x) >> 5);          // this warp in the grid
@@ -432,8 +432,6 @@ constexpr int kWalkU = 32;
 struct WalkShared {
     float2 gather[2][kMaxCluster][kWarps];   // per-warp (reference, sum) of every CTA of the cluster, by row parity
     double ctot[2][kMaxCluster];             // per-CTA totals of the final draw: [0] residual, [1] target row
-    char pad_[64];                           // keeps what follows 64 bytes into a 128-byte segment: measured, the walk is 4 % slower with the
-                                             // accept-test fields starting on a 128-byte boundary (with no padding as with 128 bytes of it)
     double dq[2];                            // the draft row's lse, by row parity
     double u[kWalkU];                        // uniforms of the accept tests of the first rows
     uint32_t pw[2], qw[2];                   // the words holding z_p(x), z_q(x) of the row's draft token
@@ -500,7 +498,7 @@ k_verify_walk(Params p, State st, Scratch sc, WalkArgs a)
 {
     constexpr int ESZ = Elem<DT>::BYTES;
     constexpr int QESZ = QP ? 4 : ESZ;
-    extern __shared__ uint4 sm_dyn[];                        // per-warp staging rings, then the partial sums of this CTA's chunks
+    extern __shared__ __align__(128) uint4 sm_dyn[];                        // per-warp staging rings, then the partial sums of this CTA's chunks
     uint4* ring = sm_dyn + (threadIdx.x >> 5) * (kStage * kVecPerLane * 32);
     float2* sm_part = reinterpret_cast<float2*>(sm_dyn + kWarps * kStage * kVecPerLane * 32);
     __shared__ WalkShared sh;
@@ -756,7 +754,7 @@ __global__ void __launch_bounds__(kThreads, kWalkResident)
 k_verify_greedy(Params p, State st, Scratch sc, WalkArgs a)
 {
     constexpr int ESZ = Elem<DT>::BYTES;
-    extern __shared__ uint4 sm_dyn[];                        // per-warp staging rings
+    extern __shared__ __align__(128) uint4 sm_dyn[];                        // per-warp staging rings
     uint4* ring = sm_dyn + (threadIdx.x >> 5) * (kStage * kVecPerLane * 32);
     __shared__ GreedyShared sh;
     cg::cluster_group cl = cg::this_cluster();
