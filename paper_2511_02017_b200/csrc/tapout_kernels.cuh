@@ -345,10 +345,13 @@ k_draft_stream(Params p, Scratch sc, StepArgs a)
 
     // Work item = (row, segment), one warp each: the first n_warps items by position in the grid, the
     // rest by ticket.  No warp ever waits for another one; the results are combined by k_draft_finish.
+    // With no more items than warps nobody needs a second one: the ticket (one address for the whole grid) is
+    // left alone.
+    const bool more = total > n_warps;
     int item = gw;
     while (item < total) {
         int nxt = 0;
-        if (lane == 0) nxt = atomicAdd(ticket, 1);       // asked for now, needed only after this item
+        if (more && lane == 0) nxt = atomicAdd(ticket, 1);       // asked for now, needed only after this item
         const int ai = item / nseg, g = item - ai * nseg;
         const int s = (FEATURES || first) ? ai : list[ai];
         const char* row = reinterpret_cast<const char*>(a.logits) + (size_t)s * a.row_stride * ESZ;
@@ -379,6 +382,7 @@ k_draft_stream(Params p, Scratch sc, StepArgs a)
             o.pad0 = o.pad1 = o.pad2 = 0;
             store_segrec(sc.seg + (size_t)s * kMaxSeg + g, o);
         }
+        if (!more) break;
         item = __shfl_sync(0xffffffffu, nxt, 0) + n_warps;
     }
     if (first) pdl_wait();
