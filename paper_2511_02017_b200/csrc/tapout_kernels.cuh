@@ -137,11 +137,22 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     const float c = a.c;
     const int pos = a.pos;
 
-    // ---- first trip, everything at once: is the sequence drafting at this position, how many rows are
-    // (the split follows from it), all segment-record slots (kMaxSeg / 32 per lane; those beyond the split are
-    // stale and masked below), chunk partials, rule state.  Nothing here waits for anything else.
+    // ---- first trip: is the sequence drafting at this position, how many rows are (the split follows from
+    // it), all segment-record slots (kMaxSeg / 32 per lane; those beyond the split are stale and masked
+    // below), chunk partials, rule state.  At position 0 every sequence drafts and everything is asked for at
+    // once; later most sequences have stopped, and two thousand warps fetching 3 KB each for nothing delay
+    // the few that need theirs, so there the question is answered first (the Philox draw fills the wait).
     const int np = FEATURES ? pos : __ldcg(sc.next_pos + s);
     const int n_rows = FEATURES ? a.n_fixed : __ldcg(sc.count + a.slot);
+    double u_draw = 0.0;
+    if (!FEATURES && ROLE != 1) u_draw = u24_to_double(rng_words(p, p.seq_offset + (uint32_t)s, a.round, (uint32_t)pos, RNG_DRAFT, 0, 0).x);
+    // (role 1 may already have moved next_pos on to pos + 1 by the time role 2 looks)
+    const bool idle = ROLE == 2 ? np < pos : np != pos;
+    if (pos > 0 && idle) {
+        // stopped at an earlier position: drafts nothing
+        if (ROLE != 2 && lane == 0 && np < pos) { a.out_token[(size_t)s * a.tok_stride] = -1; a.out_continue[s] = 0; }
+        return;
+    }
     constexpr int RPL = kMaxSeg / 32;        // segment records per lane
     SegRec r[RPL];
 #pragma unroll
@@ -156,12 +167,7 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
         sq_prev = st.sqrtH_prev[s];
         lambda = st.lambda[s];
     }
-    // the uniform of the token draw does not depend on anything loaded: worked out while the loads fly
-    double u_draw = 0.0;
-    if (!FEATURES && ROLE != 1) u_draw = u24_to_double(rng_words(p, p.seq_offset + (uint32_t)s, a.round, (uint32_t)pos, RNG_DRAFT, 0, 0).x);
-    // (role 1 may already have moved next_pos on to pos + 1 by the time role 2 looks)
-    if (ROLE == 2 ? np < pos : np != pos) {
-        // stopped at an earlier position: drafts nothing
+    if (idle) {
         if (ROLE != 2 && lane == 0 && np < pos) { a.out_token[(size_t)s * a.tok_stride] = -1; a.out_continue[s] = 0; }
         return;
     }
