@@ -248,6 +248,18 @@ def test_vocabulary_beyond_the_register_resident_chunk_table(dtype, vocab):
     torch.cuda.empty_cache()
 
 
+def test_lockstep_bench_config_all_512_rounds_sampled():
+    """Config 4 as given: batch 1024, all 512 rounds (UCB1 well past its exploration phase, AdaEDL's lambda
+    drifting for hundreds of rounds), the oracle following four of the sequences."""
+    w = si.WORKLOADS["throughput"]
+    sample = sorted(np.random.default_rng(21).choice(w.n_seq, size=4, replace=False).tolist())
+    rep, dev, _ = run_lockstep(w, w.rounds, sample=sample, device=DEV, check_state_every=16)
+    _assert_clean(rep, max_flip_rate=0.01)
+    assert rep.rounds == 512
+    dev.destroy()
+    torch.cuda.empty_cache()
+
+
 def test_million_token_vocabulary_single_cta_walk():
     """A row of 1.1 M fp32 logits walked by one CTA per sequence: 2150 chunks, so the walk's table of chunk
     partials (with its staging rings) needs more shared memory than a kernel gets without asking."""
