@@ -50,7 +50,7 @@ typedef enum {
     TAPOUT_E_ALIGNMENT = -3,    /* a logits pointer or stride is not 16-byte aligned    */
     TAPOUT_E_CUDA = -4,         /* a CUDA runtime call failed (tapout_last_cuda_error)  */
     TAPOUT_E_ALLOC = -5,        /* out of host or device memory                         */
-    TAPOUT_E_UNSUPPORTED = -6,  /* valid request this build does not implement          */
+    TAPOUT_E_UNSUPPORTED = -6,  /* valid request the library does not implement         */
     TAPOUT_E_TOO_LARGE = -7     /* more rows or a wider vocabulary than the built-in scratch of
                                    tapout_row_stats_static holds                          */
 } tapout_error;

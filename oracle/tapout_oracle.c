@@ -593,7 +593,7 @@ orc_t* orc_create(int S, int V, int K, int A, int policy, int level)
     for (int a = 0; a < A; ++a) h->rule_of_arm[a] = a % 5;   /* Table 1 order */
     h->seed = 0; h->dtype = ORC_BF16; h->inv_Tq = 1.0f; h->inv_Tp = 1.0f;
     h->rp.h_maxconf = 0.8; h->rp.h_svip = 0.6; h->rp.h_diff = 0.2; h->rp.h_margin = 0.2;
-    /* AdaEDL constants are not given in the paper; these are this build's choices. */
+    /* AdaEDL constants are not given in the paper; these are this library's choices. */
     h->rp.ada_gamma = 0.2; h->rp.ada_alpha = 0.9; h->rp.ada_beta1 = 0.5; h->rp.ada_beta2 = 0.9; h->rp.ada_eps = 0.01;
     h->ada_lambda0 = 0.4; h->ada_acc0 = 1.0;
     h->reward_alpha = 0.5; h->reward_kind = 0; h->ucb_c2 = 2.0;
