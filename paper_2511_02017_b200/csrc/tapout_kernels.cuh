@@ -130,7 +130,7 @@ __device__ __forceinline__ void store_segrec(SegRec* g, const SegRec& r) {
 // cheap first part, the row total).  Role 0 does everything in one warp (FEATURES).
 template <int DT, bool FEATURES, int ROLE>
 __device__ __forceinline__ void finish_row(const Params& p, const State& st, const Scratch& sc, const StepArgs& a, int s,
-                                           int n_warps_stream, int lane) {
+                                           int n_warps_stream, int lane, bool have_pre = false, int np_pre = 0, int n_rows_pre = 0) {
     if (!FEATURES && ROLE == 2 && p.draft_greedy) return;        // greedy decoding: the token is the argmax role 1 finds
     const char* row = reinterpret_cast<const char*>(a.logits) + (size_t)s * a.row_stride * Elem<DT>::BYTES;
     const float2* part = sc.cdf + (size_t)s * p.NC;
@@ -142,8 +142,8 @@ __device__ __forceinline__ void finish_row(const Params& p, const State& st, con
     // below), chunk partials, rule state.  At position 0 every sequence drafts and everything is asked for at
     // once; later most sequences have stopped, and two thousand warps fetching 3 KB each for nothing delay
     // the few that need theirs, so there the question is answered first (the Philox draw fills the wait).
-    const int np = FEATURES ? pos : __ldcg(sc.next_pos + s);
-    const int n_rows = FEATURES ? a.n_fixed : __ldcg(sc.count + a.slot);
+    const int np = FEATURES ? pos : have_pre ? np_pre : __ldcg(sc.next_pos + s);
+    const int n_rows = FEATURES ? a.n_fixed : have_pre ? n_rows_pre : __ldcg(sc.count + a.slot);
     double u_draw = 0.0;
     if (!FEATURES && ROLE != 1) u_draw = u24_to_double(rng_words(p, p.seq_offset + (uint32_t)s, a.round, (uint32_t)pos, RNG_DRAFT, 0, 0).x);
     // (role 1 may already have moved next_pos on to pos + 1 by the time role 2 looks)
@@ -335,13 +335,15 @@ k_draft_stream(Params p, Scratch sc, StepArgs a)
     const int lane = threadIdx.x & 31;
     const int gw = (int)((blockIdx.x * kThreads + threadIdx.x) >> 5);          // this warp in the grid
     const int n_warps = (int)((gridDim.x * kThreads) >> 5);
-    pdl_trigger();
     // Position 0 reads nothing its predecessors in the stream write (every sequence drafts, in index order;
     // the ticket was zeroed by the last finish kernel), so it starts at once and overlaps the tail of the
     // previous round's verification and its update; it waits for them only before it exits, which is what
-    // the finish kernel behind it relies on.
+    // the finish kernel behind it relies on.  Later positions wait first and let their successor go after
+    // that: the finish kernel behind them then starts only once the previous finish kernel has completed,
+    // and may read what that one wrote (who drafts, how many rows) while this kernel is still streaming.
     const bool first = !FEATURES && a.pos == 0;
     if (!first) pdl_wait();
+    pdl_trigger();
     int* ticket = sc.count + 4;
     const int n_rows = FEATURES ? a.n_fixed : first ? p.S : sc.count[a.slot];
     const int32_t* list = sc.list + (size_t)a.slot * p.S;
@@ -406,6 +408,12 @@ k_draft_finish(Params p, State st, Scratch sc, StepArgs a, int n_warps_stream)
     const int gw = (int)((blockIdx.x * kFinishThreads + threadIdx.x) >> 5);
     const int n_warps = (int)((gridDim.x * kFinishThreads) >> 5);
     pdl_trigger();
+    // At positions >= 1 this kernel starts only after the previous finish kernel has completed (see
+    // k_draft_stream), and the streaming kernel in between writes neither of these: whether the sequence
+    // drafts here and how many rows do are fetched while that kernel is still at work.
+    const bool have_pre = !FEATURES && a.pos > 0 && (gw >> 1) < p.S;
+    int np_pre = 0, n_rows_pre = 0;
+    if (have_pre) { np_pre = __ldcg(sc.next_pos + (gw >> 1)); n_rows_pre = __ldcg(sc.count + a.slot); }
     pdl_wait();
     if (gw == 0 && lane == 0) {
         sc.count[4] = 0;                                 // the work ticket of the next streaming kernel
@@ -416,8 +424,9 @@ k_draft_finish(Params p, State st, Scratch sc, StepArgs a, int n_warps_stream)
     } else {
         // two warps per sequence: even warps the features and the rule, odd warps the token
         for (int s = gw >> 1; s < p.S; s += n_warps >> 1) {
-            if (gw & 1) finish_row<DT, false, 2>(p, st, sc, a, s, n_warps_stream, lane);
-            else finish_row<DT, false, 1>(p, st, sc, a, s, n_warps_stream, lane);
+            const bool pre = have_pre && s == (gw >> 1);
+            if (gw & 1) finish_row<DT, false, 2>(p, st, sc, a, s, n_warps_stream, lane, pre, np_pre, n_rows_pre);
+            else finish_row<DT, false, 1>(p, st, sc, a, s, n_warps_stream, lane, pre, np_pre, n_rows_pre);
         }
     }
 }
