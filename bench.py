@@ -204,7 +204,8 @@ def bench_ours(args):
     POOL_ROUNDS = args.pool_rounds
     S, K, V = w.n_seq, w.k_max, w.vocab
     # weak scaling: every rank owns a full-size shard of independent sequences, ids offset by rank
-    dev = tp.Tapout.from_workload(w, seq_offset=rank * S, token_out_stride=K, **variant_params(args))
+    # the logits of every round are generated and synchronised before the timed region: position 0 may start early
+    dev = tp.Tapout.from_workload(w, seq_offset=rank * S, token_out_stride=K, early_start=0 if args.no_early_start else 1, **variant_params(args))
     if args.row_segments:
         dev.set_param("row_segments", args.row_segments)
     if args.verify_cluster:
@@ -331,7 +332,10 @@ def bench_ours(args):
                        "rows_per_step": rows / args.steps, "row_bytes": row_bytes,
                        "l2_policy": "inputs larger than L2: %d rounds of %.2f GB cycled" %
                                     (POOL_ROUNDS, (2 * K + 1) * S * row_bytes / 1e9),
-                       "sharding": "independent sequences per GPU, no collective" if world > 1 else "single GPU"},
+                       "sharding": "independent sequences per GPU, no collective" if world > 1 else "single GPU",
+                       "schedule": ("every kernel waits for its predecessor" if args.no_early_start else
+                                    "early_start: every round's logits are resident and synchronised before the timed "
+                                    "region, so position 0 of a round may start under the previous round's verification")},
             "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "roofline": roofline, "kernels": kernels,
             "rows": {"draft": rows_d, "target": rows_t, "residual": rows_r},
             "rows_lifetime": {"draft": life["rows_draft"], "target": life["rows_target"], "residual": life["rows_residual"]},
@@ -395,6 +399,7 @@ def main():
     ap.add_argument("--row-segments", type=int, default=0, help="CTAs per draft row (0 = library default)")
     ap.add_argument("--verify-cluster", type=int, default=0, help="CTAs per verify cluster (0 = library default)")
     ap.add_argument("--pool-rounds", type=int, default=POOL_ROUNDS)
+    ap.add_argument("--no-early-start", action="store_true", help="position 0 waits for the previous round like every other kernel")
     ap.add_argument("--greedy", action="store_true", help="greedy draft + verification by matching the target's top token")
     args = ap.parse_args()
     if args.impl == "reference":

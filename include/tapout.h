@@ -112,7 +112,13 @@ typedef enum {
                                       instead of a draw; features and stop rule unchanged (default 0)        */
     TAPOUT_P_VERIFY_GREEDY = 35,   /* i64: 1 = tapout_verify accepts by matching the target's top token (see there; default 0) */
     TAPOUT_P_Q_FORMAT = 36,        /* i64: what tapout_verify's draft_probs holds: TAPOUT_Q_LOGITS (default) or TAPOUT_Q_PROBS_F32 */
-    TAPOUT_P__COUNT = 37
+    TAPOUT_P_EARLY_START = 37,     /* i64: 1 = the caller vouches that the draft logits of position 0 of every round are complete
+                                      and visible before the call that reads them is made (produced earlier and synchronised,
+                                      not by work still queued ahead of the call on the handle's stream).  The streaming kernel
+                                      of position 0 then does not wait for what precedes it in the stream and overlaps the
+                                      previous round's verification and update.  0 (default) = it waits like every other kernel.
+                                      Scheduling only: results do not depend on it                                          */
+    TAPOUT_P__COUNT = 38
 } tapout_param;
 
 /* Values of TAPOUT_P_Q_FORMAT. */

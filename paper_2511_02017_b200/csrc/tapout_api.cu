@@ -47,6 +47,7 @@ struct tapout {
     int grid_rows = 0;
     int cluster_user = 0, cluster = 1;   // CTAs per verify cluster: requested (0 = automatic) and in use
     size_t walk_smem = 0;
+    bool staging = false;                // inside tapout_round_host: the logits are copied in just ahead of the kernels
     bool q_probs = false;                // tapout_verify's draft tensor holds fp32 probabilities, not logits
     bool arms_ready = false;             // the arms of round `round` are chosen and the round's lists are set up
     // host-round staging
@@ -256,10 +257,12 @@ int draft_step_impl(tapout* h, const void* logits, int64_t stride, int32_t* out_
     if (h->profile) h->prof_n[0] += 2;
     const unsigned fin_grid = (unsigned)((2 * (long long)h->p.S + 3) / 4);    // two warps per sequence, four per CTA
     const int n_warps = h->grid_rows * kWarps;
-    const size_t ring_bytes = sizeof(uint4) * kWarps * kStage * kVecPerLane * 32;   // position 0 loads straight into registers
+    const size_t ring_bytes = sizeof(uint4) * kWarps * kStage * kVecPerLane * 32;
+    Params ps = h->p;
+    if (h->staging) ps.early_start = 0;                    // the copies that bring the rows in are still queued ahead of this launch   // position 0 loads straight into registers
     TP_CUDA(h, h->p.dtype == DT_BF16
-                   ? launch_chained(k_draft_stream<DT_BF16, false>, h->grid_rows, kThreads, ring_bytes, h->stream, 0, h->p, h->sc, a)
-                   : launch_chained(k_draft_stream<DT_FP32, false>, h->grid_rows, kThreads, ring_bytes, h->stream, 0, h->p, h->sc, a));
+                   ? launch_chained(k_draft_stream<DT_BF16, false>, h->grid_rows, kThreads, ring_bytes, h->stream, 0, ps, h->sc, a)
+                   : launch_chained(k_draft_stream<DT_FP32, false>, h->grid_rows, kThreads, ring_bytes, h->stream, 0, ps, h->sc, a));
     TP_LAUNCHED(h);
     TP_CUDA(h, h->p.dtype == DT_BF16
                    ? launch_chained(k_draft_finish<DT_BF16, false>, fin_grid, kFinishThreads, 0, h->stream, 0, h->p, h->st, h->sc, a, n_warps)
@@ -367,7 +370,7 @@ int tapout_create(tapout_t** out, int n_seq, int vocab, int k_max, int n_arms, i
     p.ada_gamma = 0.2; p.ada_alpha = 0.9; p.ada_beta1 = 0.5; p.ada_beta2 = 0.9; p.ada_eps = 0.01;
     p.ada_lambda0 = 0.4; p.ada_acc0 = 1.0;
     p.reward_alpha = 0.5; p.ucb_c2 = 2.0; p.ts_mu0 = 0.0; p.ts_var0 = 1.0; p.ts_noise_var = 1.0;
-    p.ts_a0 = 1; p.ts_b0 = 1; p.reward_kind = 0; p.token_update_all = 1; p.draft_greedy = 0; p.verify_greedy = 0;
+    p.ts_a0 = 1; p.ts_b0 = 1; p.reward_kind = 0; p.token_update_all = 1; p.draft_greedy = 0; p.verify_greedy = 0; p.early_start = 0;
     h->step_stride = vocab;
     h->q_seq = (int64_t)k_max * vocab; h->q_pos = vocab;
     h->p_seq = (int64_t)(k_max + 1) * vocab; h->p_pos = vocab;
@@ -450,6 +453,7 @@ int tapout_set_param_i64(tapout_t* h, int key, int64_t v) {
     case TAPOUT_P_TOKEN_UPDATE_ALL: p.token_update_all = v ? 1 : 0; return TAPOUT_OK;
     case TAPOUT_P_DRAFT_GREEDY: p.draft_greedy = v ? 1 : 0; return TAPOUT_OK;
     case TAPOUT_P_VERIFY_GREEDY: p.verify_greedy = v ? 1 : 0; return TAPOUT_OK;
+    case TAPOUT_P_EARLY_START: p.early_start = v ? 1 : 0; return TAPOUT_OK;
     case TAPOUT_P_Q_FORMAT: if (v != TAPOUT_Q_LOGITS && v != TAPOUT_Q_PROBS_F32) return TAPOUT_E_INVALID_ARG; h->q_probs = v == TAPOUT_Q_PROBS_F32; return TAPOUT_OK;
     case TAPOUT_P_TOKEN_OUT_STRIDE: if (v < 1) return TAPOUT_E_INVALID_ARG; h->tok_stride = v; return TAPOUT_OK;
     case TAPOUT_P_PROFILE: h->profile = v != 0; return TAPOUT_OK;
@@ -520,6 +524,7 @@ int tapout_get_param_i64(const tapout_t* h, int key, int64_t* v) {
     case TAPOUT_P_TOKEN_UPDATE_ALL: *v = p.token_update_all; return TAPOUT_OK;
     case TAPOUT_P_DRAFT_GREEDY: *v = p.draft_greedy; return TAPOUT_OK;
     case TAPOUT_P_VERIFY_GREEDY: *v = p.verify_greedy; return TAPOUT_OK;
+    case TAPOUT_P_EARLY_START: *v = p.early_start; return TAPOUT_OK;
     case TAPOUT_P_Q_FORMAT: *v = h->q_probs ? TAPOUT_Q_PROBS_F32 : TAPOUT_Q_LOGITS; return TAPOUT_OK;
     case TAPOUT_P_ROW_SEGMENTS: *v = p.nseg; return TAPOUT_OK;
     case TAPOUT_P_VERIFY_CLUSTER: *v = h->cluster; return TAPOUT_OK;
@@ -635,6 +640,7 @@ int tapout_round_host(tapout_t* h, const void* draft_logits, const void* target_
     const size_t rb = V * esz;                                            // bytes of one row
     std::vector<int> active(S), n_drafted(S, 0);
     for (size_t s2 = 0; s2 < S; ++s2) active[s2] = (int)s2;
+    struct Staging { tapout* h; explicit Staging(tapout* h_) : h(h_) { h->staging = true; } ~Staging() { h->staging = false; } } staging(h);
     TP_CUDA(h, cudaMemsetAsync(d_tok, 0xff, 4 * S * K, h->stream));        // -1 beyond the drafted length
     for (int i = 0; i < p.K && !active.empty(); ++i) {
         if (active.size() * 4 >= S) {                                     // most rows: one strided copy of the position

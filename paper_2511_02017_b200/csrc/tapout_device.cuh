@@ -38,6 +38,7 @@ struct Params {
     uint32_t ts_a0, ts_b0;
     int reward_kind, token_update_all;
     int draft_greedy, verify_greedy;     // greedy decoding of the draft; verification by matching the target's top token
+    int early_start;                     // position 0 may start before its predecessors in the stream have completed
     int nseg, NC;                        // CTAs per draft row, chunks per row
 };
 

@@ -342,7 +342,10 @@ k_draft_stream(Params p, Scratch sc, StepArgs a)
     // that: the finish kernel behind them then starts only once the previous finish kernel has completed,
     // and may read what that one wrote (who drafts, how many rows) while this kernel is still streaming.
     const bool first = !FEATURES && a.pos == 0;
-    if (!first) pdl_wait();
+    // (only when the caller has vouched for the logits of position 0 being complete and visible before the call:
+    // a kernel that skips the wait may start before whatever precedes it in the stream has finished writing)
+    const bool early = first && p.early_start;
+    if (!early) pdl_wait();
     pdl_trigger();
     int* ticket = sc.count + 4;
     const int n_rows = FEATURES ? a.n_fixed : first ? p.S : sc.count[a.slot];
@@ -393,7 +396,7 @@ k_draft_stream(Params p, Scratch sc, StepArgs a)
         if (!more) break;
         item = __shfl_sync(0xffffffffu, nxt, 0) + n_warps;
     }
-    if (first) pdl_wait();
+    if (early) pdl_wait();
 }
 
 // Second kernel of a draft position: two warps per sequence (finish_row, roles 1 and 2; a sequence that is not drafting

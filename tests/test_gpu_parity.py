@@ -489,13 +489,17 @@ def test_round_call_matches_separate_calls():
     b.destroy()
 
 
+@pytest.mark.parametrize("early_start", [1, 0])
 @pytest.mark.parametrize("n_seq,vocab", [(96, 20008), (7, 4104), (300, 2056)])
-def test_rounds_back_to_back_without_synchronising(n_seq, vocab):
-    """Rounds enqueued with nothing between them (position 0 of a round then overlaps the previous round's
-    verification tail and update) give what the same rounds give with a synchronisation after every call."""
+def test_rounds_back_to_back_without_synchronising(n_seq, vocab, early_start):
+    """Rounds enqueued with nothing between them give what the same rounds give with a synchronisation after
+    every call -- also with early_start, where position 0 of a round overlaps the previous round's
+    verification tail and update (all logits here exist before the first call)."""
     w = si.scaled(si.WORKLOADS["throughput"], n_seq=n_seq, vocab=vocab)
     from tests.lockstep import make_device
-    a, b = make_device(w), make_device(w, token_out_stride=w.k_max)   # b's steps write column i of the token matrix
+    a = make_device(w, early_start=early_start)
+    b = make_device(w, token_out_stride=w.k_max)                      # b's steps write column i of the token matrix
+    assert a.get_param("early_start") == early_start and b.get_param("early_start") == 0
     S, K, R = w.n_seq, w.k_max, 12
     pool = [peaked_logits(w, r, DEV) for r in range(R)]
     mk = lambda shape, dt: [torch.zeros(shape, dtype=dt, device=DEV) for _ in range(R)]
