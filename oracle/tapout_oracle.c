@@ -446,7 +446,9 @@ void orc_verify_sequence(const void* q_rows, long q_pos_stride, const void* p_ro
         Z += res[v];
     }
     if (Z > 0.0) {
-        out->next_token = orc_sample_cdf(res, V, Z, u2, tol, &out->next_lo, &out->next_hi);
+        /* the band of acceptable draws is tol in probability units around u2 * Z (the residual entries are
+         * probabilities, and the deciding quantity, their running sum, is one): tol / Z as a fraction of Z */
+        out->next_token = orc_sample_cdf(res, V, Z, u2, tol / Z, &out->next_lo, &out->next_hi);
     } else {
         out->zero_residual = 1;
         out->next_token = orc_sample_cdf(wp, V, sp.W, u2, tol, &out->next_lo, &out->next_hi);
@@ -499,7 +501,9 @@ void orc_verify_sequence_qprobs(const float* q_rows, long q_pos_stride, const vo
         Z += res[v];
     }
     if (Z > 0.0) {
-        out->next_token = orc_sample_cdf(res, V, Z, u2, tol, &out->next_lo, &out->next_hi);
+        /* the band of acceptable draws is tol in probability units around u2 * Z (the residual entries are
+         * probabilities, and the deciding quantity, their running sum, is one): tol / Z as a fraction of Z */
+        out->next_token = orc_sample_cdf(res, V, Z, u2, tol / Z, &out->next_lo, &out->next_hi);
     } else {
         out->zero_residual = 1;
         out->next_token = orc_sample_cdf(wp, V, sp.W, u2, tol, &out->next_lo, &out->next_hi);

@@ -108,3 +108,31 @@ def test_engine_uses_the_probabilities():
         assert v["accept_len"][s] == a
         if a < K:
             assert v["next_token"][s] != toks[s, a]                  # the residual is p with the drafted token removed
+
+
+def test_residual_band_is_measured_in_probability():
+    """The set of acceptable residual draws is what a running sum off by 1e-6 of probability could give: with a
+    residual mass of 1e-3 that is a thousandth of the mass, not a millionth."""
+    p = np.array([0.4, 0.3, 0.3, 0.0])
+    q = np.array([[0.3994, 0.2996, 0.3, 0.001]], np.float32)        # residual [6e-4, 4e-4, 0, 0]; token 3 is always rejected
+    P = np.tile(_logits_from_probs(p), (2, 1))
+    seen = set()
+    for seq in range(40000):
+        u = orc.rng_uniform(5, seq, 0, 0, orc.RNG_RESAMPLE)
+        if 0.6002 < u < 0.6008:
+            kind, want = "just above", (1, 0, 1)
+        elif 0.5992 < u < 0.5998:
+            kind, want = "just below", (0, 0, 1)
+        elif 0.30 < u < 0.31:
+            kind, want = "far", (0, 0, 0)
+        elif 0.80 < u < 0.81:
+            kind, want = "far above", (1, 1, 1)
+        else:
+            continue
+        out = orc.verify_sequence_qprobs(q, P, [3], seed=5, seq=seq, rnd=0)
+        assert out.accept_len == 0
+        assert (out.next_token, out.next_lo, out.next_hi) == want, (kind, u)
+        seen.add(kind)
+        if len(seen) == 4:
+            break
+    assert len(seen) == 4
