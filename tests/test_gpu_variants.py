@@ -211,3 +211,45 @@ def test_arm_report_runs_every_controller():
     assert 1.0 <= r["mean_drafted"] <= 6.0 and r["plays"] == [12 * 6]
     r = arm_report.run(w, 10, si.peaked_round_logits, DEV, 5, "ts", "token")
     assert len(r["plays"]) == 5 and sum(r["plays"]) >= 12 * 10 and 1.0 <= r["rows_per_token"] <= 3.0
+
+
+# ------------------------------------------------------------------ random shapes, controllers and variants
+def test_random_shapes_controllers_and_variants():
+    """A seeded sweep of small cases: vocabularies from one vector to 70 000 tokens, 1 ... 257 sequences, k_max
+    1 ... 16, 1 ... 16 arms with random rules, every controller, both dtypes, temperatures, both rewards, forced
+    cluster sizes and row splits, flat and peaked rows, and the three variants of the verification step."""
+    rng = np.random.default_rng(7)
+    total, flips = 0, 0
+    for case in range(150):
+        dtype = str(rng.choice(["bf16", "fp32"]))
+        mult = 8 if dtype == "bf16" else 4
+        V = int(rng.choice([mult, 3 * mult, 520, 1032, 2056, 4104, 9000 // mult * mult, 20008, 33000 // mult * mult,
+                            70000 // mult * mult]))
+        S = int(rng.choice([1, 2, 3, 7, 16, 33, 100, 257]))
+        K = int(rng.choice([1, 2, 3, 5, 8, 16]))
+        A = int(rng.choice([1, 2, 3, 5, 8, 16]))
+        policy, level = str(rng.choice(["ucb1", "ts", "ucb_tuned"])), str(rng.choice(["seq", "token"]))
+        sigma = str(rng.choice(["fixed:0.5", "per_seq:0.1:1.5", "per_round:0.2:2.0"]))
+        w = si.Workload("rnd", S, V, dtype, K, 1, A, policy, level, seed=int(rng.integers(0, 1 << 30)), sigma=sigma,
+                        temp_draft=float(rng.choice([1.0, 0.8])), temp_target=float(rng.choice([1.0, 0.7, 1.3])),
+                        c=float(rng.choice([1.0, 0.8])))
+        variant = str(rng.choice(["plain", "plain", "greedy", "vgreedy", "qprobs"]))
+        params = {"plain": {}, "greedy": GREEDY, "vgreedy": dict(verify_greedy=1), "qprobs": QPROBS}[variant]
+        extra, oextra = {}, {}
+        if rng.random() < 0.3:
+            extra["verify_cluster"] = int(rng.choice([1, 2, 4, 8]))
+        if rng.random() < 0.3:
+            extra["row_segments"] = int(rng.choice([1, 2, 7, 64]))
+        if rng.random() < 0.3:
+            extra["reward_kind"] = oextra["reward_kind"] = 1
+        arms = [int(x) for x in rng.integers(0, 6, A)]
+        gen = si.peaked_round_logits if rng.random() < 0.7 and V >= 64 else si.round_logits
+        sample = None if S <= 33 else sorted(rng.choice(S, size=12, replace=False).tolist())
+        rep, dev, _ = run_lockstep(w, int(rng.integers(2, 6)), sample=sample, device=DEV, logits_fn=gen,
+                                   dev_params=dict(arms=arms, **params, **extra), orc_params=dict(arms=arms, **params, **oextra))
+        dev.destroy()
+        assert rep.ok() and rep.max_feat_err <= 1e-5, (case, w, variant, extra, arms, rep.summary(), rep.failures[:3])
+        total += sum(rep.decisions.values())
+        flips += sum(rep.flips.values())
+    assert flips <= 0.001 * total, (flips, total)
+    torch.cuda.empty_cache()
