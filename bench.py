@@ -249,6 +249,28 @@ def bench_ours(args):
     rows_all, ms_all = aggregate(rows, ms, world, backend_ready)
     value = rows_all / (ms_all * 1e-3)
 
+    # ---- the same loop with every kernel waiting for its predecessor (the library's default schedule)
+    strict = None
+    if not args.no_early_start:
+        dev.set_param("early_start", 0)
+        n_strict = max(1, min(args.steps, 100))
+        for r in range(4):
+            step(r)
+        torch.cuda.synchronize()
+        ss0 = dev.get_status()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record()
+        for r in range(n_strict):
+            step(4 + r)
+        s1.record()
+        torch.cuda.synchronize()
+        ss1 = dev.get_status()
+        rows_s = sum(ss1[k] - ss0[k] for k in ("rows_draft", "rows_target", "rows_residual"))
+        rows_s_all, ms_s_all = aggregate(rows_s, s0.elapsed_time(s1), world, backend_ready)
+        strict = {"value": rows_s_all / (ms_s_all * 1e-3), "unit": UNIT, "steps": n_strict, "ms_per_step": ms_s_all / n_strict,
+                  "schedule": "every kernel waits for its predecessor (early_start off)"}
+        dev.set_param("early_start", 1)
+
     # ---- per-kernel device time (separate pass, same steps, event intervals per kernel class)
     dev.set_param("profile", 1)
     for k in range(3):
@@ -340,6 +362,7 @@ def bench_ours(args):
             "rows": {"draft": rows_d, "target": rows_t, "residual": rows_r},
             "rows_lifetime": {"draft": life["rows_draft"], "target": life["rows_target"], "residual": life["rows_residual"]},
             "hbm_gbs": rows * row_bytes / (ms * 1e-3) / 1e9,
+            "strict_schedule": strict,
             "cpu_baseline": cpu,
         }
         print(json.dumps(line))
