@@ -400,10 +400,12 @@ def test_checkpoint_resume_is_bitwise_equivalent():
     c.destroy()
 
 
-def test_round_host_matches_device_path():
+@pytest.mark.parametrize("early_start", [0, 1])
+def test_round_host_matches_device_path(early_start):
+    """(with early_start set as well: the host path copies its rows in just ahead of the kernels and must not use it)"""
     w = si.Workload("host", 5, 4104, "bf16", 4, 1, 5, "ucb1", "seq", seed=41)
     from tests.lockstep import make_device
-    a, b = make_device(w), make_device(w)
+    a, b = make_device(w), make_device(w, early_start=early_start)
     S, K = w.n_seq, w.k_max
     tok = torch.empty(S, dtype=torch.int32, device=DEV)
     cont = torch.empty(S, dtype=torch.uint8, device=DEV)
