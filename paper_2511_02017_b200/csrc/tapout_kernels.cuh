@@ -30,14 +30,18 @@ constexpr int kWalkResident = 5;          // k_verify_walk CTAs resident per SM 
 // Into how many segments a draft row is cut, one warp per segment, decided on the device from the number
 // of rows actually drafted at this position (the host never learns it).  Many rows: about three items per
 // warp of the grid so that the ticket counter can even out slow and fast SMs, but segments of at least
-// six chunks so that a segment's epilogue stays small beside its streaming.  Few rows: as many segments
-// as it takes to give every warp of the grid something to read, down to one chunk per segment.
+// six chunks so that a segment's epilogue stays small beside its streaming.  Fewer rows than an eighth of
+// the grid's warps: as many segments as give every warp at most one item, down to two chunks per segment.
 __device__ __forceinline__ int segments_for(const Params& p, int n_rows, int n_warps) {
     const int cap = max(1, min(kMaxSeg, p.NC));
     if (p.nseg > 0) return min(p.nseg, cap);
     if (n_rows <= 0) return 1;
+    // Few enough rows that every warp of the grid can have an item of at most NC / 8 chunks: exactly one item per
+    // warp or none (rounded down: one segment more per row would leave a handful of warps with a second item
+    // and double the kernel's length).
+    const int one_wave = n_warps / n_rows;
+    if (one_wave >= 8) return max(1, min(one_wave, cap));
     int nseg = min((3 * n_warps + n_rows - 1) / n_rows, max(p.NC / 6, 1));
-    if ((long long)n_rows * nseg < n_warps) nseg = (n_warps + n_rows - 1) / n_rows;
     return max(1, min(nseg, cap));
 }
 
